@@ -1,0 +1,207 @@
+/*
+ * Oracle: Algorithm 1 (Slow Momentum) with the base-optimizer directions of Table C.1,
+ * one coordinate j at a time. TEST INFRASTRUCTURE: see slowmo_oracle.h.
+ *
+ * This file is compiled twice: with -DORACLE_F64=0 (binary32, the parity gate) and with
+ * -DORACLE_F64=1 (binary64, for the pins). Built with -ffp-contract=off; every fused
+ * operation is an explicit FMA(), every other operation rounds once in `real`.
+ *
+ * Readings where the paper leaves a choice (each also listed in the design notes):
+ *  - Table C.1's Adam step count l: 1-based number of Adam steps since the buffers were
+ *    last zeroed (the caption's l = k or l = t tau + k would divide by 1 - beta^0 = 0).
+ *    Under the "average" policy buffers are not zeroed, so l keeps counting.
+ *  - Weight decay is L2: added to the gradient before the momentum update.
+ *  - The buffer policy of outer iteration t+1 is applied right after the outer update
+ *    of iteration t (at t = 0 every policy is a no-op because the buffers are zero).
+ *  - 1/gamma_t and alpha*gamma_t are formed once per outer iteration (in binary64,
+ *    rounded once to `real`); the worker sum runs in worker order 0..m-1 and is divided
+ *    by m.
+ */
+#include "slowmo_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#if ORACLE_F64
+typedef double real;
+#define FMA(a, b, c) fma((a), (b), (c))
+#define SQRT(a) sqrt(a)
+#define RUN_NAME slowmo_oracle_run_f64
+#else
+typedef float real;
+#define FMA(a, b, c) fmaf((a), (b), (c))
+#define SQRT(a) sqrtf(a)
+#define RUN_NAME slowmo_oracle_run_f32
+#endif
+
+/* Stochastic gradient of worker i at coordinate j, step (t,k), evaluated at x. */
+static real gradient(const oracle_config *cfg, uint32_t i, uint64_t j, uint32_t t, uint32_t k,
+                     real x, real a_j, real c_ij, real G_ij) {
+  real g;
+  if (cfg->grad_mode == ORACLE_GRAD_GENERATED) {
+    /* F_i(x) = 1/2 sum_j a_j (x_j - c_{i,j})^2, gradient a_j (x_j - c_{i,j}), plus sigma z */
+    uint64_t key = oracle_stream_key(ORACLE_TAG_GRADNOISE, cfg->seed, t, k, i);
+    real z = (real)oracle_word_to_normal(oracle_stream_word(key, j));
+    real noise = (real)cfg->sigma * z;
+    real e = x - c_ij;
+    g = FMA(a_j, e, noise);
+  } else {
+    g = G_ij;
+  }
+  if (cfg->weight_decay != 0.0f) g = FMA((real)cfg->weight_decay, x, g);
+  return g;
+}
+
+static int valid(const oracle_config *c) {
+  if (c->m == 0 || c->tau == 0) return 0;
+  if (c->base != ORACLE_BASE_NESTEROV && c->base != ORACLE_BASE_ADAM) return 0;
+  if (c->buffer_policy < ORACLE_BUF_RESET || c->buffer_policy > ORACLE_BUF_AVERAGE) return 0;
+  if (c->grad_mode < ORACLE_GRAD_GENERATED || c->grad_mode > ORACLE_GRAD_SUPPLIED_ARRAY) return 0;
+  return 1;
+}
+
+int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_idx, uint64_t j0,
+             uint64_t n, const float *G, real *x_out, real *anchor_out, real *u_out, real *h_out,
+             real *v_out, double *dbar) {
+  if (!cfg || !valid(cfg) || !x_out || !anchor_out || !u_out || !h_out) return -1;
+  if (cfg->grad_mode == ORACLE_GRAD_SUPPLIED_ARRAY && !G) return -1;
+  const uint32_t m = cfg->m, tau = cfg->tau, T = cfg->T;
+  const int adam = cfg->base == ORACLE_BASE_ADAM;
+  const real mu = (real)cfg->mu;
+  const real b1 = (real)cfg->adam_b1, b2 = (real)cfg->adam_b2, eps = (real)cfg->adam_eps;
+  const real omb1 = (real)(1.0 - (double)cfg->adam_b1); /* 1 - beta_1 */
+  const real omb2 = (real)(1.0 - (double)cfg->adam_b2); /* 1 - beta_2 */
+  const real alpha = (real)cfg->alpha, beta = (real)cfg->beta;
+  (void)alpha;
+
+#pragma omp parallel
+  {
+    real *x = (real *)malloc(sizeof(real) * m);
+    real *h = (real *)malloc(sizeof(real) * m);
+    real *v = (real *)malloc(sizeof(real) * m);
+    real *c = (real *)malloc(sizeof(real) * m);
+    real *Gfix = (real *)malloc(sizeof(real) * m);
+
+#pragma omp for schedule(static)
+    for (uint64_t q = 0; q < n; ++q) {
+      const uint64_t j = j_idx ? j_idx[q] : j0 + q;
+
+      /* synthetic problem data of this coordinate */
+      real a_j = 0;
+      for (uint32_t i = 0; i < m; ++i) c[i] = Gfix[i] = 0;
+      if (cfg->grad_mode == ORACLE_GRAD_GENERATED) {
+        a_j = (real)oracle_curvature(cfg, j);
+        for (uint32_t i = 0; i < m; ++i) c[i] = (real)oracle_centre(cfg, i, j);
+      } else if (cfg->grad_mode == ORACLE_GRAD_SUPPLIED_HASH) {
+        for (uint32_t i = 0; i < m; ++i) Gfix[i] = (real)oracle_supplied_gradient(cfg, i, j);
+      }
+
+      /* Algorithm 1, input line: all workers start at x_{0,0}; u_0 = 0; buffers are zero */
+      real x0 = (real)cfg->x_init; /* anchor x_{t,0} */
+      real u = 0;
+      for (uint32_t i = 0; i < m; ++i) {
+        x[i] = x0;
+        h[i] = 0;
+        v[i] = 0;
+      }
+      uint64_t l = 0;            /* Adam steps since the buffers were last zero */
+      double pow_b1 = 1.0, pow_b2 = 1.0; /* beta_1^l, beta_2^l */
+
+      for (uint32_t t = 0; t < T; ++t) {
+        const double gam_d = (double)(gamma_t ? gamma_t[t] : cfg->gamma);
+        const real gam = (real)gam_d;
+        const real inv_gam = (real)(1.0 / gam_d);
+        const real alpha_gam = (real)((double)cfg->alpha * gam_d);
+
+        for (uint32_t k = 0; k < tau; ++k) {
+          l += 1;
+          pow_b1 *= (double)cfg->adam_b1;
+          pow_b2 *= (double)cfg->adam_b2;
+          const real ibc1 = (real)(1.0 / (1.0 - pow_b1)); /* 1 / (1 - beta_1^l) */
+          const real ibc2 = (real)(1.0 / (1.0 - pow_b2)); /* 1 / (1 - beta_2^l) */
+          double dsum = 0.0;
+
+          for (uint32_t i = 0; i < m; ++i) {
+            real G_ij = Gfix[i];
+            if (cfg->grad_mode == ORACLE_GRAD_SUPPLIED_ARRAY)
+              G_ij = (real)G[(((uint64_t)t * tau + k) * m + i) * n + q];
+            const real g = gradient(cfg, i, j, t, k, x[i], a_j, c[i], G_ij);
+            real d;
+            if (!adam) {
+              /* Table C.1, SGD row: h <- mu h + g ; d = mu h + g (Nesterov momentum) */
+              h[i] = FMA(mu, h[i], g);
+              d = FMA(mu, h[i], g);
+            } else {
+              /* Table C.1, Adam row */
+              h[i] = FMA(b1, h[i], omb1 * g);
+              v[i] = FMA(b2, v[i], omb2 * (g * g));
+              const real h_hat = h[i] * ibc1;
+              const real v_hat = v[i] * ibc2;
+              d = h_hat / (SQRT(v_hat) + eps);
+            }
+            /* Algorithm 1, base optimizer step: x_{t,k+1} = x_{t,k} - gamma_t d */
+            x[i] = FMA(-gam, d, x[i]);
+            dsum += (double)d;
+          }
+          if (dbar) dbar[((uint64_t)t * tau + k) * n + q] = dsum / (double)m;
+        }
+
+        /* Algorithm 1, exact average over the workers */
+        real s = x[0];
+        for (uint32_t i = 1; i < m; ++i) s = s + x[i];
+        const real xbar = s / (real)m;
+        /* Eq. (2): u_{t+1} = beta u_t + (x_{t,0} - xbar_{t,tau}) / gamma_t */
+        u = FMA(beta, u, (x0 - xbar) * inv_gam);
+        /* Eq. (3): x_{t+1,0} = x_{t,0} - alpha gamma_t u_{t+1} */
+        x0 = FMA(-alpha_gam, u, x0);
+        /* every worker continues from x_{t+1,0} */
+        for (uint32_t i = 0; i < m; ++i) x[i] = x0;
+
+        /* buffer policy for the next outer iteration */
+        if (cfg->buffer_policy == ORACLE_BUF_RESET) {
+          for (uint32_t i = 0; i < m; ++i) h[i] = v[i] = 0;
+          l = 0;
+          pow_b1 = pow_b2 = 1.0;
+        } else if (cfg->buffer_policy == ORACLE_BUF_AVERAGE) {
+          real sh = h[0], sv = v[0];
+          for (uint32_t i = 1; i < m; ++i) {
+            sh = sh + h[i];
+            sv = sv + v[i];
+          }
+          const real hbar = sh / (real)m, vbar = sv / (real)m;
+          for (uint32_t i = 0; i < m; ++i) {
+            h[i] = hbar;
+            v[i] = vbar;
+          }
+        } /* maintain: nothing */
+      }
+
+      for (uint32_t i = 0; i < m; ++i) {
+        x_out[(uint64_t)i * n + q] = x[i];
+        h_out[(uint64_t)i * n + q] = h[i];
+        if (v_out) v_out[(uint64_t)i * n + q] = v[i];
+      }
+      anchor_out[q] = x0;
+      u_out[q] = u;
+    }
+    free(x);
+    free(h);
+    free(v);
+    free(c);
+    free(Gfix);
+  }
+  return 0;
+}
+
+#if !ORACLE_F64
+int slowmo_oracle_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+#endif
