@@ -1,0 +1,211 @@
+/*
+ * libslowmo: the data-parallel hot path of Slow Momentum (SlowMo; Wang, Tantia, Ballas,
+ * Rabbat, ICLR 2020) for m simulated workers held as an [m, P] fp32 replica tensor on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library runs the two phases of the paper's Algorithm 1:
+ *   - the inner loop: tau steps x <- x - gamma_t d of the base optimizer on every replica,
+ *     with the directions d of Table C.1 (SGD with Nesterov momentum, or Adam);
+ *   - the outer step: exact average over the replicas, slow-momentum update (Eq. 2),
+ *     outer-iterate update (Eq. 3), broadcast to all replicas, and the reset / maintain /
+ *     average policy for the base-optimizer buffers (first statement of the outer loop).
+ *
+ * Conventions for every entry point
+ *   Memory     All tensors are DEVICE pointers owned by the caller and borrowed for the
+ *              life of the context. The library never allocates or frees tensor memory.
+ *              slowmo_create makes one small device allocation (a status block of a few
+ *              words) that slowmo_destroy releases.
+ *   Layout     Row-major fp32. 2-D tensors are [m, pitch]: row i (worker i) starts at
+ *              base + i*pitch elements; columns P..pitch-1 are padding. 1-D tensors have
+ *              pitch elements. pitch is a multiple of 4 and >= P; every base pointer is
+ *              16-byte aligned. Kernels process whole 4-element column groups, so padding
+ *              columns below the next multiple of 4 are computed on and hold unspecified
+ *              finite-or-not values; they are never returned by slowmo_get_params.
+ *   Stream     Work is enqueued on the CUDA stream given at creation; calls return without
+ *              waiting unless stated. One context per stream; a context is not thread-safe.
+ *   Errors     Every call returns a SLOWMO_* status; nothing aborts or throws. CUDA
+ *              failures are sticky in the context (SLOWMO_ECUDA; the cudaError_t is
+ *              available from slowmo_last_cuda_error).
+ *   Numerics   All arithmetic is IEEE binary32 with the operation order documented at each
+ *              call; the same configuration and seed give bit-identical state on every run.
+ */
+#ifndef SLOWMO_H
+#define SLOWMO_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct slowmo_ctx slowmo_ctx;
+
+enum {
+  SLOWMO_OK = 0,
+  SLOWMO_EINVAL = -1,   /* bad argument (value, enum, NULL)                         */
+  SLOWMO_ESTATE = -2,   /* call not legal at this point of Algorithm 1              */
+  SLOWMO_EALIGN = -3,   /* pointer not 16-byte aligned or pitch not a multiple of 4 */
+  SLOWMO_ECUDA = -4,    /* a CUDA call failed; sticky                               */
+  SLOWMO_ENOMEM = -5,   /* host allocation failed                                   */
+  SLOWMO_ETIMEOUT = -6, /* a bounded device-side wait gave up                       */
+  SLOWMO_ENOTIMPL = -7
+};
+enum { SLOWMO_BASE_NESTEROV = 0, SLOWMO_BASE_ADAM = 1 };
+enum { SLOWMO_BUF_RESET = 0, SLOWMO_BUF_MAINTAIN = 1, SLOWMO_BUF_AVERAGE = 2 };
+enum { SLOWMO_GRAD_GENERATED = 0, SLOWMO_GRAD_SUPPLIED = 1 };
+/* tensors addressable by slowmo_get_params / slowmo_set_params */
+enum {
+  SLOWMO_T_X = 0,      /* replicas x^{(i)}            [m, pitch] */
+  SLOWMO_T_ANCHOR = 1, /* x_{t,0}                     [pitch]    */
+  SLOWMO_T_U = 2,      /* slow momentum u_t           [pitch]    */
+  SLOWMO_T_H = 3,      /* first buffer h^{(i)}        [m, pitch] */
+  SLOWMO_T_V = 4,      /* Adam second moment v^{(i)}  [m, pitch] */
+  SLOWMO_T_A = 5,      /* curvature a_j               [pitch]    (generated mode) */
+  SLOWMO_T_C = 6       /* centres c_{i,j}             [m, pitch] (generated mode) */
+};
+/* kernels whose implementation can be selected with slowmo_set_variant */
+enum { SLOWMO_K_LOCAL = 0, SLOWMO_K_OUTER = 1 };
+enum {
+  SLOWMO_VARIANT_DEFAULT = 0,
+  SLOWMO_OUTER_DIRECT = 1, /* vector loads straight to registers                      */
+  SLOWMO_OUTER_STAGED = 2  /* bulk-copy (TMA) staging of row tiles through shared mem  */
+};
+
+/*
+ * Problem statement, after the "Input" line of Algorithm 1 (base optimizer with learning
+ * rate gamma_t, tau, alpha, beta, m, x_{0,0}; u_0 = 0) plus the synthetic objective used in
+ * generated-gradient mode: worker i minimises 1/2 sum_j a_j (x_j - c_{i,j})^2 and sees the
+ * stochastic gradient a_j (x_j - c_{i,j}) + sigma z, z ~ N(0,1) from a counter-based hash of
+ * (seed, t, k, i, j). a_j ~ U[a_lo, a_hi), c_{i,j} ~ N(0, c_std^2) are drawn from the same
+ * hash at creation.
+ */
+typedef struct {
+  uint64_t P;   /* parameters per replica (> 0)                                  */
+  uint32_t m;   /* workers / replicas (> 0)                                      */
+  uint32_t tau; /* base-optimizer steps per outer iteration (> 0)                */
+  float alpha;  /* slow learning rate (> 0)                                      */
+  float beta;   /* slow momentum factor, in [0, 1)                               */
+  float gamma;  /* base learning rate gamma_0 (> 0, finite); see slowmo_set_gamma */
+  int32_t base; /* SLOWMO_BASE_*                                                 */
+  float mu;           /* beta_local of Table C.1 (SGD row), in [0, 1)            */
+  float weight_decay; /* L2 coefficient, added to the gradient: g <- g + wd x    */
+  float adam_b1, adam_b2, adam_eps; /* Table C.1 (Adam row); betas in [0,1), eps > 0 */
+  int32_t buffer_policy;            /* SLOWMO_BUF_*                              */
+  int32_t grad_mode;                /* SLOWMO_GRAD_*                             */
+  uint64_t seed;
+  float a_lo, a_hi, c_std, sigma; /* generator constants (sigma also scales slowmo_fill_gradient) */
+  float x_init;                   /* x_{0,0} in every coordinate                 */
+  uint32_t n_tensors;             /* optional segment table: number of parameter tensors */
+  const uint64_t *tensor_sizes;   /* HOST array of n_tensors sizes summing to P, or NULL */
+} slowmo_config;
+
+/* Device tensors borrowed from the caller (see "Layout" above). */
+typedef struct {
+  float *x;       /* [m, pitch]                                         */
+  float *h;       /* [m, pitch]                                         */
+  float *v;       /* [m, pitch]; required for Adam, may be NULL else    */
+  float *anchor;  /* [pitch]                                            */
+  float *u;       /* [pitch]                                            */
+  float *a;       /* [pitch];    required in generated mode, else NULL  */
+  float *c;       /* [m, pitch]; required in generated mode, else NULL  */
+  uint64_t pitch; /* row length in elements                             */
+} slowmo_buffers;
+
+/*
+ * Create a context and initialise the state of Algorithm 1's input line on the stream:
+ * x^{(i)} = anchor = x_init, u = 0, h = v = 0, and in generated mode a and c from the hash.
+ * `cuda_stream` is a cudaStream_t (NULL = the legacy default stream).
+ * Errors: EINVAL (any constraint listed beside the fields, unknown enum, NULL pointer,
+ * sizes not summing to P), EALIGN, ENOMEM, ECUDA.
+ */
+int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cuda_stream,
+                  slowmo_ctx **out);
+
+/* Release the context (never the caller's tensors). Waits for the stream first. */
+int slowmo_destroy(slowmo_ctx *ctx);
+
+/*
+ * Inner loop of Algorithm 1: n base-optimizer steps on all m replicas, one fused kernel
+ * launch per step. With k the steps already taken in this outer iteration, k + n <= tau is
+ * required (ESTATE otherwise).
+ *
+ * Per element (worker i, coordinate j), in binary32:
+ *   gradient   generated: e = x - c ; g = fma(a, e, sigma*z(t,k,i,j))   supplied: g = grad[i,j]
+ *              then, if weight_decay != 0, g = fma(wd, x, g)
+ *   Nesterov   h = fma(mu, h, g) ; d = fma(mu, h, g)                       (Table C.1, SGD)
+ *   Adam       h = fma(b1, h, (1-b1)*g) ; v = fma(b2, v, (1-b2)*(g*g)) ;
+ *              d = (h * 1/(1-b1^l)) / (sqrt(v * 1/(1-b2^l)) + eps)         (Table C.1, Adam)
+ *              l = Adam steps since the buffers were last zero (1-based)
+ *   step       x = fma(-gamma_t, d, x)                                     (Algorithm 1)
+ *
+ * `grad` is a device [m, pitch] tensor in supplied mode (read by each of the n steps) and
+ * must be NULL in generated mode (EINVAL otherwise).
+ */
+int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad);
+
+/*
+ * Outer step of Algorithm 1 in one fused kernel; legal only after exactly tau local steps
+ * (ESTATE otherwise). Per coordinate j, in binary32, with the gamma_t of this iteration:
+ *   average    s = x^{(0)} ; s = s + x^{(i)} for i = 1..m-1 in order ; xbar = s / m
+ *   Eq. (2)    u = fma(beta, u, (anchor - xbar) * (1/gamma_t))
+ *   Eq. (3)    anchor = fma(-(alpha*gamma_t), u, anchor)
+ *   broadcast  x^{(i)} = anchor for every i
+ *   buffers    reset: h = v = 0 and l = 0; maintain: untouched;
+ *              average: h^{(i)} = (sum over i in order) / m for every i, same for v
+ * 1/gamma_t and alpha*gamma_t are formed in binary64 on the host and rounded once.
+ * Advances the outer counter t and sets k = 0.
+ */
+int slowmo_outer_step(slowmo_ctx *ctx);
+
+/* Change the base learning rate (a schedule's gamma_t). Legal only between outer
+ * iterations, i.e. when k = 0 (ESTATE otherwise). EINVAL unless gamma > 0 and finite. */
+int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t);
+
+/*
+ * Copy out part of a tensor: columns [offset, offset+count) of row `replica` (or of every
+ * row when replica = -1, giving a dense [m, count] result; replica must be -1 or 0 for 1-D
+ * tensors). offset + count <= P. `dst` is a host pointer (the call then waits for the
+ * stream) or, with dst_on_device != 0, a device pointer (the copy is enqueued).
+ */
+int slowmo_get_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count,
+                      float *dst, int dst_on_device);
+
+/* Inverse of slowmo_get_params: overwrite part of a tensor from host or device memory.
+ * Used to restore a checkpoint and to upload per-worker problem data. */
+int slowmo_set_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count,
+                      const float *src, int src_on_device);
+
+/* Position in Algorithm 1: outer iteration t, inner steps k taken in it, Adam count l. */
+int slowmo_get_counters(slowmo_ctx *ctx, uint64_t *t, uint32_t *k, uint64_t *l);
+
+/* Fill a device [m, pitch] tensor with the fixed synthetic gradient G[i,j] = sigma * z from
+ * the hash (stream tag 5, worker i). For supplied-mode benchmarks; enqueued on the stream. */
+int slowmo_fill_gradient(slowmo_ctx *ctx, float *grad);
+
+/*
+ * Export n consecutive draws of one noise stream, coordinates j0 <= j < j0 + n: the raw
+ * 64-bit words (SplitMix64 outputs) and/or the binary32 normals derived from them.
+ * Either device pointer may be NULL. Tags: 1 curvature, 2 centres, 3 gradient noise,
+ * 5 supplied gradient. Test hook for the bit-exact comparison of the integer stream.
+ */
+int slowmo_debug_noise(slowmo_ctx *ctx, uint32_t tag, uint64_t t, uint32_t k, uint32_t w, uint64_t j0,
+                       uint64_t n, uint64_t *words, float *normals);
+
+/* Segment idx of the optional parameter-tensor table: first coordinate and length. */
+int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_t *count);
+
+/* Select the implementation of a kernel (SLOWMO_K_*, SLOWMO_VARIANT_* / SLOWMO_OUTER_*);
+ * all variants compute identical results. */
+int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant);
+
+/* Wait for the stream and report SLOWMO_ETIMEOUT if any kernel recorded that one of its
+ * bounded waits ran out (the record is then cleared), SLOWMO_ECUDA on a CUDA failure. */
+int slowmo_sync_status(slowmo_ctx *ctx);
+
+const char *slowmo_strerror(int status);
+int slowmo_last_cuda_error(slowmo_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

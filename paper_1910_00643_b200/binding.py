@@ -1,0 +1,275 @@
+"""ctypes binding of libslowmo.so: the same entry points as include/slowmo.h, argument
+marshalling only. PyTorch is used for device memory and streams; every step of the method
+runs in the library's CUDA kernels.
+
+There is no fallback: if the shared library is missing or a call fails, an exception is
+raised.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libslowmo.so")
+
+OK, EINVAL, ESTATE, EALIGN, ECUDA, ENOMEM, ETIMEOUT, ENOTIMPL = 0, -1, -2, -3, -4, -5, -6, -7
+BASE = {"nesterov": 0, "adam": 1}
+POLICY = {"reset": 0, "maintain": 1, "average": 2}
+GRAD = {"generated": 0, "supplied": 1}
+TENSOR = {"x": 0, "anchor": 1, "u": 2, "h": 3, "v": 4, "a": 5, "c": 6}
+KERNEL = {"local": 0, "outer": 1}
+VARIANT = {"default": 0, "direct": 1, "staged": 2}
+EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_outer_step",
+           "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
+           "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
+           "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error"]
+
+
+class SlowMoError(RuntimeError):
+    def __init__(self, status, what):
+        self.status = status
+        super().__init__(f"{what}: {strerror(status)} ({status})")
+
+
+class Config(C.Structure):
+    _fields_ = [
+        ("P", C.c_uint64), ("m", C.c_uint32), ("tau", C.c_uint32),
+        ("alpha", C.c_float), ("beta", C.c_float), ("gamma", C.c_float),
+        ("base", C.c_int32), ("mu", C.c_float), ("weight_decay", C.c_float),
+        ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
+        ("buffer_policy", C.c_int32), ("grad_mode", C.c_int32),
+        ("seed", C.c_uint64),
+        ("a_lo", C.c_float), ("a_hi", C.c_float), ("c_std", C.c_float), ("sigma", C.c_float),
+        ("x_init", C.c_float),
+        ("n_tensors", C.c_uint32), ("tensor_sizes", C.POINTER(C.c_uint64)),
+    ]
+
+
+class Buffers(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("h", C.c_void_p), ("v", C.c_void_p), ("anchor", C.c_void_p),
+                ("u", C.c_void_p), ("a", C.c_void_p), ("c", C.c_void_p), ("pitch", C.c_uint64)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libslowmo.so (once). Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_1910_00643_b200.build` (needs nvcc)")
+        L = C.CDLL(LIB_PATH)
+        vp, u64, u32, i32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32
+        sig = {
+            "slowmo_create": [C.POINTER(Config), C.POINTER(Buffers), vp, C.POINTER(vp)],
+            "slowmo_destroy": [vp],
+            "slowmo_local_steps": [vp, u32, vp],
+            "slowmo_outer_step": [vp],
+            "slowmo_set_gamma": [vp, C.c_float],
+            "slowmo_get_params": [vp, C.c_int, i32, u64, u64, vp, C.c_int],
+            "slowmo_set_params": [vp, C.c_int, i32, u64, u64, vp, C.c_int],
+            "slowmo_get_counters": [vp, C.POINTER(u64), C.POINTER(u32), C.POINTER(u64)],
+            "slowmo_fill_gradient": [vp, vp],
+            "slowmo_debug_noise": [vp, u32, u64, u32, u32, u64, u64, vp, vp],
+            "slowmo_tensor_range": [vp, u32, C.POINTER(u64), C.POINTER(u64)],
+            "slowmo_set_variant": [vp, C.c_int, C.c_int],
+            "slowmo_sync_status": [vp],
+            "slowmo_last_cuda_error": [vp],
+        }
+        for name, args in sig.items():
+            f = getattr(L, name)
+            f.argtypes = args
+            f.restype = C.c_int
+        L.slowmo_strerror.argtypes = [C.c_int]
+        L.slowmo_strerror.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def strerror(status):
+    return lib().slowmo_strerror(status).decode()
+
+
+def _check(status, what):
+    if status != OK:
+        raise SlowMoError(status, what)
+
+
+def make_config(*, P, m, tau, alpha=1.0, beta=0.0, gamma=0.1, base="nesterov", mu=0.0, weight_decay=0.0,
+                adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, buffer_policy="reset", grad_mode="generated",
+                seed=0, a_lo=0.5, a_hi=2.0, c_std=1.0, sigma=0.0, x_init=0.0, tensor_sizes=None, **_ignored):
+    """Fill the C config from paper-notation keyword arguments (see include/slowmo.h)."""
+    cfg = Config(P, m, tau, alpha, beta, gamma, BASE[base] if isinstance(base, str) else base, mu,
+                 weight_decay, adam_b1, adam_b2, adam_eps,
+                 POLICY[buffer_policy] if isinstance(buffer_policy, str) else buffer_policy,
+                 GRAD[grad_mode] if isinstance(grad_mode, str) else grad_mode, seed, a_lo, a_hi, c_std,
+                 sigma, x_init, 0, None)
+    if tensor_sizes is not None:
+        arr = (C.c_uint64 * len(tensor_sizes))(*[int(s) for s in tensor_sizes])
+        cfg._keep = arr
+        cfg.n_tensors = len(tensor_sizes)
+        cfg.tensor_sizes = C.cast(arr, C.POINTER(C.c_uint64))
+    return cfg
+
+
+def round_up(n, q):
+    return (n + q - 1) // q * q
+
+
+class SlowMo:
+    """One SlowMo context with its device tensors (torch-allocated) on the current device.
+
+    Methods carry the names of the C entry points without the prefix and do nothing but
+    marshal arguments.
+    """
+
+    def __init__(self, workload, stream=None, pitch=None, guard=0):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("libslowmo needs a CUDA device (sm_100a); there is no CPU path")
+        self.torch = torch
+        w = dict(workload)
+        if w.get("n_tensors") and "tensor_sizes" not in w:
+            from .workloads import tensor_sizes
+            w["tensor_sizes"] = tensor_sizes(w["P"], w["n_tensors"], w.get("seed", 0))
+        self.workload = w
+        self.cfg = make_config(**w)
+        self.P, self.m, self.tau = w["P"], w["m"], w["tau"]
+        self.pitch = pitch if pitch is not None else round_up(self.P, 32)
+        self.stream = stream if stream is not None else torch.cuda.Stream()
+        self.guard = guard
+        adam = self.cfg.base == BASE["adam"]
+        generated = self.cfg.grad_mode == GRAD["generated"]
+        self._raw = {}
+        self.t = {}
+        for name, rows, need in (("x", self.m, True), ("h", self.m, True), ("v", self.m, adam),
+                                 ("anchor", 1, True), ("u", 1, True), ("a", 1, generated),
+                                 ("c", self.m, generated)):
+            self.t[name] = self._alloc(name, rows) if need else None
+        ptr = lambda k: self.t[k].data_ptr() if self.t[k] is not None else None
+        self.buf = Buffers(ptr("x"), ptr("h"), ptr("v"), ptr("anchor"), ptr("u"), ptr("a"), ptr("c"), self.pitch)
+        self.grad = None
+        self.ctx = C.c_void_p()
+        # creation enqueues fills on self.stream; order it after the allocations' stream
+        self.stream.wait_stream(torch.cuda.current_stream())
+        _check(lib().slowmo_create(C.byref(self.cfg), C.byref(self.buf), self.stream.cuda_stream,
+                                   C.byref(self.ctx)), "slowmo_create")
+
+    # guard words before and after every tensor let tests detect out-of-bounds writes
+    GUARD_VALUE = -12345.5
+
+    def _alloc(self, name, rows):
+        torch = self.torch
+        n = rows * self.pitch
+        g = self.guard
+        raw = torch.empty(n + 2 * g, dtype=torch.float32, device="cuda")
+        if g:
+            raw[:g] = self.GUARD_VALUE
+            raw[g + n:] = self.GUARD_VALUE
+        self._raw[name] = raw
+        return raw[g:g + n]
+
+    def guards_intact(self):
+        g = self.guard
+        self.synchronize()
+        for name, raw in self._raw.items():
+            n = raw.numel() - 2 * g
+            if g and not (bool((raw[:g] == self.GUARD_VALUE).all()) and bool((raw[g + n:] == self.GUARD_VALUE).all())):
+                return False
+        return True
+
+    def alloc_gradient(self):
+        """Device [m, pitch] tensor for supplied-gradient mode (kept as self.grad)."""
+        self.grad = self._alloc("grad", self.m)
+        return self.grad
+
+    def fill_gradient(self, grad=None):
+        grad = self.grad if grad is None else grad
+        _check(lib().slowmo_fill_gradient(self.ctx, grad.data_ptr()), "slowmo_fill_gradient")
+
+    def local_steps(self, n, grad=None):
+        _check(lib().slowmo_local_steps(self.ctx, n, None if grad is None else grad.data_ptr()),
+               "slowmo_local_steps")
+
+    def outer_step(self):
+        _check(lib().slowmo_outer_step(self.ctx), "slowmo_outer_step")
+
+    def set_gamma(self, gamma):
+        _check(lib().slowmo_set_gamma(self.ctx, gamma), "slowmo_set_gamma")
+
+    def set_variant(self, kernel, variant):
+        _check(lib().slowmo_set_variant(self.ctx, KERNEL[kernel], VARIANT[variant]), "slowmo_set_variant")
+
+    def sync_status(self):
+        _check(lib().slowmo_sync_status(self.ctx), "slowmo_sync_status")
+
+    def counters(self):
+        t, k, l = C.c_uint64(), C.c_uint32(), C.c_uint64()
+        _check(lib().slowmo_get_counters(self.ctx, C.byref(t), C.byref(k), C.byref(l)), "slowmo_get_counters")
+        return t.value, k.value, l.value
+
+    def get_params(self, which, replica=-1, offset=0, count=None, out=None):
+        """Copy columns [offset, offset+count) of tensor `which` to host (numpy) or to `out`
+        (a torch CUDA tensor or pinned/pageable numpy array)."""
+        count = self.P - offset if count is None else count
+        rows = 1 if (replica >= 0 or which in ("anchor", "u", "a")) else self.m
+        on_device = 0
+        if out is None:
+            out = np.empty((rows, count), np.float32)
+            dst = out.ctypes.data
+        elif isinstance(out, np.ndarray):
+            dst = out.ctypes.data
+        else:
+            dst = out.data_ptr()
+            on_device = 1 if out.is_cuda else 0
+        _check(lib().slowmo_get_params(self.ctx, TENSOR[which], replica, offset, count, dst, on_device),
+               "slowmo_get_params")
+        return out
+
+    def set_params(self, which, src, replica=-1, offset=0, count=None):
+        count = self.P - offset if count is None else count
+        if isinstance(src, np.ndarray):
+            assert src.dtype == np.float32 and src.flags.c_contiguous
+            ptr, on_device = src.ctypes.data, 0
+        else:
+            ptr, on_device = src.data_ptr(), 1 if src.is_cuda else 0
+        _check(lib().slowmo_set_params(self.ctx, TENSOR[which], replica, offset, count, ptr, on_device),
+               "slowmo_set_params")
+
+    def debug_noise(self, tag, t, k, w, j0, n, words=True, normals=True):
+        torch = self.torch
+        with torch.cuda.stream(self.stream):
+            wd = torch.empty(n, dtype=torch.int64, device="cuda") if words else None
+            z = torch.empty(n, dtype=torch.float32, device="cuda") if normals else None
+        _check(lib().slowmo_debug_noise(self.ctx, tag, t, k, w, j0, n, wd.data_ptr() if words else None,
+                                        z.data_ptr() if normals else None), "slowmo_debug_noise")
+        self.synchronize()
+        return (wd.cpu().numpy().view(np.uint64) if words else None, z.cpu().numpy() if normals else None)
+
+    def tensor_range(self, idx):
+        off, cnt = C.c_uint64(), C.c_uint64()
+        _check(lib().slowmo_tensor_range(self.ctx, idx, C.byref(off), C.byref(cnt)), "slowmo_tensor_range")
+        return off.value, cnt.value
+
+    def run(self, T, grad=None):
+        """T outer iterations of Algorithm 1: tau local steps, then the outer step."""
+        for _ in range(T):
+            self.local_steps(self.tau, grad)
+            self.outer_step()
+
+    def synchronize(self):
+        self.stream.synchronize()
+
+    def close(self):
+        if self.ctx:
+            _check(lib().slowmo_destroy(self.ctx), "slowmo_destroy")
+            self.ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

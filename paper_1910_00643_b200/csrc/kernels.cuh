@@ -1,0 +1,257 @@
+// sm_100a kernels of the SlowMo hot path: synthetic-input fills, the fused multi-replica
+// base-optimizer step (Algorithm 1's inner statement with Table C.1's directions) and the
+// fused outer step (exact average, Eq. 2, Eq. 3, broadcast, buffer policy).
+//
+// All of them are HBM-bound streams over [m, pitch] fp32 tensors: one 128-bit access per
+// thread per tensor, full-line coalescing across the warp, several independent loads in
+// flight per thread, and grids of many short blocks so the tail is negligible.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "noise.cuh"
+
+namespace slowmo {
+
+constexpr int kThreads = 256;
+
+// ---- streaming 128-bit accesses --------------------------------------------------------
+// Tensors are far larger than L2 and every line is used exactly once per launch, so loads
+// and stores carry the evict-first policy.
+__device__ __forceinline__ float4 ld_stream(const float *p) { return __ldcs(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ void st_stream(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
+// `a` is shared by the m rows of a column tile: keep it cacheable so the blocks of the other
+// rows, which run next to this one, find it in L2.
+__device__ __forceinline__ float4 ld_shared_row(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+
+__device__ __forceinline__ float &comp(float4 &v, int e) { return reinterpret_cast<float *>(&v)[e]; }
+__device__ __forceinline__ float comp(const float4 &v, int e) { return reinterpret_cast<const float *>(&v)[e]; }
+
+// ---- K0: fills ---------------------------------------------------------------------------
+
+// dst[i, j] = scale * z(tag, seed, 0, 0, i, j) for every row i and column j < 4*nvec.
+__global__ void __launch_bounds__(kThreads)
+fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t tag, uint64_t seed, float scale) {
+  const uint32_t row = blockIdx.y;
+  const uint64_t key = stream_key(tag, seed, 0, 0, row);
+  float *p = dst + (uint64_t)row * pitch;
+  for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
+    uint64_t s = key + kGoldenGamma * (4 * vi + 1);
+    float4 o;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      comp(o, e) = __fmul_rn(scale, word_to_normal(mix64(s)));
+      s += kGoldenGamma;
+    }
+    st_stream(p + 4 * vi, o);
+  }
+}
+
+// a[j] = fma(a_hi - a_lo, U_j, a_lo), U_j from the curvature stream.
+__global__ void __launch_bounds__(kThreads)
+fill_curvature_kernel(float *a, uint32_t nvec, uint64_t seed, float a_lo, float a_hi) {
+  const uint64_t key = stream_key(kTagCurvature, seed, 0, 0, 0);
+  const float span = __fsub_rn(a_hi, a_lo);
+  for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
+    uint64_t s = key + kGoldenGamma * (4 * vi + 1);
+    float4 o;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      comp(o, e) = __fmaf_rn(span, word_to_unit(mix64(s)), a_lo);
+      s += kGoldenGamma;
+    }
+    st_stream(a + 4 * vi, o);
+  }
+}
+
+// dst[i, j] = value for every row and column j < 4*nvec.
+__global__ void __launch_bounds__(kThreads)
+fill_value_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, float value) {
+  float *p = dst + (uint64_t)blockIdx.y * pitch;
+  const float4 o = make_float4(value, value, value, value);
+  for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads)
+    st_stream(p + 4 * vi, o);
+}
+
+// Export of one stream for the bit-exact test: words and/or normals for j0 <= j < j0 + n.
+__global__ void __launch_bounds__(kThreads)
+export_stream_kernel(uint64_t key, uint64_t j0, uint64_t n, uint64_t *words, float *normals) {
+  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (uint64_t)gridDim.x * kThreads) {
+    const uint64_t r = stream_word(key, j0 + i);
+    if (words) words[i] = r;
+    if (normals) normals[i] = word_to_normal(r);
+  }
+}
+
+// ---- K1: fused multi-replica base-optimizer step ------------------------------------------
+
+struct LocalArgs {
+  float *x, *h, *v;       // [m, pitch]
+  const float *src;       // generated mode: centres c [m, pitch]; supplied mode: gradient G [m, pitch]
+  const float *a;         // [pitch], generated mode
+  uint64_t pitch;
+  uint32_t nvec;          // 4-element column groups per row
+  uint32_t m;
+  uint64_t seed, t;       // outer iteration, for the noise key
+  uint32_t k;             // inner step, for the noise key
+  float neg_gamma, mu, wd, sigma;
+  float b1, b2, omb1, omb2, ibc1, ibc2, eps;  // Adam: betas, 1-betas, 1/(1-beta^l), epsilon
+};
+
+// One block = one tile of kThreads*U column groups of one row. Consecutive blocks are the m
+// rows of the same tile, so the shared curvature tile is read from DRAM once and from L2
+// m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic.
+template <int BASE, int GRAD, int U>
+__global__ void __launch_bounds__(kThreads)
+local_step_kernel(const LocalArgs A) {
+  const uint32_t row = blockIdx.x % A.m;
+  const uint32_t tile = blockIdx.x / A.m;
+  const uint32_t v0 = tile * (uint32_t)(kThreads * U) + threadIdx.x;
+  const uint64_t roff = (uint64_t)row * A.pitch;
+
+  __shared__ uint64_t key_sh;
+  if (GRAD == 0) {
+    if (threadIdx.x == 0) key_sh = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
+    __syncthreads();
+  }
+
+  float4 x[U], h[U], v[U], s[U], a[U];
+  bool ok[U];
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    const uint32_t vi = v0 + u * kThreads;
+    ok[u] = vi < A.nvec;
+    if (ok[u]) {
+      const uint64_t off = roff + 4ull * vi;
+      x[u] = ld_stream(A.x + off);
+      h[u] = ld_stream(A.h + off);
+      if (BASE == 1) v[u] = ld_stream(A.v + off);
+      s[u] = ld_stream(A.src + off);
+      if (GRAD == 0) a[u] = ld_shared_row(A.a + 4ull * vi);
+    }
+  }
+
+#pragma unroll
+  for (int u = 0; u < U; ++u) {
+    if (!ok[u]) continue;
+    const uint32_t vi = v0 + u * kThreads;
+    uint64_t st = 0;
+    if (GRAD == 0) st = key_sh + kGoldenGamma * (4ull * vi + 1);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float xe = comp(x[u], e);
+      float g;
+      if (GRAD == 0) {
+        const float z = word_to_normal(mix64(st));
+        st += kGoldenGamma;
+        g = __fmaf_rn(comp(a[u], e), __fsub_rn(xe, comp(s[u], e)), __fmul_rn(A.sigma, z));
+      } else {
+        g = comp(s[u], e);
+      }
+      if (A.wd != 0.0f) g = __fmaf_rn(A.wd, xe, g);
+      float d;
+      if (BASE == 0) {
+        const float hn = __fmaf_rn(A.mu, comp(h[u], e), g);
+        d = __fmaf_rn(A.mu, hn, g);
+        comp(h[u], e) = hn;
+      } else {
+        const float hn = __fmaf_rn(A.b1, comp(h[u], e), __fmul_rn(A.omb1, g));
+        const float vn = __fmaf_rn(A.b2, comp(v[u], e), __fmul_rn(A.omb2, __fmul_rn(g, g)));
+        const float hh = __fmul_rn(hn, A.ibc1);
+        const float vh = __fmul_rn(vn, A.ibc2);
+        d = __fdiv_rn(hh, __fadd_rn(__fsqrt_rn(vh), A.eps));
+        comp(h[u], e) = hn;
+        comp(v[u], e) = vn;
+      }
+      comp(x[u], e) = __fmaf_rn(A.neg_gamma, d, xe);
+    }
+    const uint64_t off = roff + 4ull * vi;
+    st_stream(A.x + off, x[u]);
+    st_stream(A.h + off, h[u]);
+    if (BASE == 1) st_stream(A.v + off, v[u]);
+  }
+}
+
+// ---- K2: fused outer step, direct variant ---------------------------------------------------
+
+struct OuterArgs {
+  float *x, *h, *v;   // [m, pitch]
+  float *anchor, *u;  // [pitch]
+  uint64_t pitch;
+  uint32_t nvec, m;
+  float beta, inv_gamma, neg_alpha_gamma, m_float;
+};
+
+// Sum of the m rows of one column group in row order, then division by m. ROWS loads are
+// issued together; the additions stay in index order.
+template <int ROWS>
+__device__ __forceinline__ float4 ordered_row_mean(const float *base, uint64_t pitch, uint32_t m, float m_float) {
+  float4 s = ld_stream(base);
+  uint32_t i = 1;
+  for (; i + ROWS <= m; i += ROWS) {
+    float4 r[ROWS];
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) r[q] = ld_stream(base + (uint64_t)(i + q) * pitch);
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) {
+      s.x = __fadd_rn(s.x, r[q].x);
+      s.y = __fadd_rn(s.y, r[q].y);
+      s.z = __fadd_rn(s.z, r[q].z);
+      s.w = __fadd_rn(s.w, r[q].w);
+    }
+  }
+  for (; i < m; ++i) {
+    const float4 r = ld_stream(base + (uint64_t)i * pitch);
+    s.x = __fadd_rn(s.x, r.x);
+    s.y = __fadd_rn(s.y, r.y);
+    s.z = __fadd_rn(s.z, r.z);
+    s.w = __fadd_rn(s.w, r.w);
+  }
+  return make_float4(__fdiv_rn(s.x, m_float), __fdiv_rn(s.y, m_float), __fdiv_rn(s.z, m_float),
+                     __fdiv_rn(s.w, m_float));
+}
+
+__device__ __forceinline__ void store_rows(float *base, uint64_t pitch, uint32_t m, float4 val) {
+#pragma unroll 4
+  for (uint32_t i = 0; i < m; ++i) st_stream(base + (uint64_t)i * pitch, val);
+}
+
+// One thread = one 4-element column group: rows in, (u, anchor) update, rows out.
+// NBUF = number of base-optimizer buffers (1: h, 2: h and v); POLICY as SLOWMO_BUF_*.
+template <int NBUF, int POLICY>
+__global__ void __launch_bounds__(kThreads)
+outer_step_direct_kernel(const OuterArgs A) {
+  const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
+  if (vi >= A.nvec) return;
+  const uint64_t col = 4ull * vi;
+
+  const float4 x0 = ld_stream(A.anchor + col);
+  const float4 u0 = ld_stream(A.u + col);
+  const float4 xbar = ordered_row_mean<8>(A.x + col, A.pitch, A.m, A.m_float);
+  float4 un, xn;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    // Eq. (2): u <- beta u + (x_{t,0} - xbar)/gamma ; Eq. (3): x_{t+1,0} <- x_{t,0} - alpha gamma u
+    const float ue = __fmaf_rn(A.beta, comp(u0, e), __fmul_rn(__fsub_rn(comp(x0, e), comp(xbar, e)), A.inv_gamma));
+    comp(un, e) = ue;
+    comp(xn, e) = __fmaf_rn(A.neg_alpha_gamma, ue, comp(x0, e));
+  }
+  st_stream(A.u + col, un);
+  st_stream(A.anchor + col, xn);
+  store_rows(A.x + col, A.pitch, A.m, xn);
+
+  if (POLICY == 0) {  // reset
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    store_rows(A.h + col, A.pitch, A.m, zero);
+    if (NBUF == 2) store_rows(A.v + col, A.pitch, A.m, zero);
+  } else if (POLICY == 2) {  // average
+    const float4 hbar = ordered_row_mean<8>(A.h + col, A.pitch, A.m, A.m_float);
+    store_rows(A.h + col, A.pitch, A.m, hbar);
+    if (NBUF == 2) {
+      const float4 vbar = ordered_row_mean<8>(A.v + col, A.pitch, A.m, A.m_float);
+      store_rows(A.v + col, A.pitch, A.m, vbar);
+    }
+  }
+}
+
+}  // namespace slowmo

@@ -1,0 +1,263 @@
+// K2, staged variant: the fused outer step of Algorithm 1 (exact average, Eq. 2, Eq. 3,
+// broadcast, buffer policy) with the replica rows moved by the bulk-copy engine (TMA).
+//
+// A persistent CTA owns column tiles of kTileCols columns. For each tile a producer thread
+// streams the m row segments into a ring of shared-memory stages with
+// cp.async.bulk (global -> shared, completion on an mbarrier); eight consumer warps add the
+// rows in worker order, apply Eq. (2)/(3), put the new anchor tile in shared memory once and
+// one thread sends it to all m replica rows (and the anchor) with m+1 bulk stores
+// (shared -> global). The buffer policy reuses the same machinery: "reset" bulk-stores a
+// zero tile, "average" streams the h (and v) rows through the ring like x.
+//
+// No cluster multicast is used anywhere; every copy is CTA-local and starts on a 16-byte
+// boundary (tile starts are multiples of kTileCols, pitch is a multiple of 4, tile widths
+// are multiples of 4 elements).
+//
+// Every mbarrier wait is bounded. A wait that runs out records SLOWMO_ETIMEOUT data in the
+// status block, raises a CTA-wide abort flag and the CTA finishes its loops without further
+// copies or global writes, then waits (bounded) for the copies it still has in flight.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels.cuh"
+
+namespace slowmo {
+
+constexpr int kTileCols = 1024;                    // columns per tile: 4 per consumer thread
+constexpr int kStageRows = 4;                      // row segments per pipeline stage
+constexpr int kStages = 6;                         // ring depth
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kStagedThreads = kConsumerThreads + 32;  // + one producer warp
+constexpr uint32_t kWaitTries = 1u << 20;          // bound of every mbarrier wait
+constexpr int kStagedCtasPerSm = 2;
+
+struct StagedSmem {
+  float stage[kStages][kStageRows][kTileCols];
+  float out[2][kTileCols];
+  float zeros[kTileCols];
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  volatile int abort;
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(void *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void *bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait. Returns immediately once the CTA is aborting; on exhaustion records where.
+__device__ __forceinline__ void mbar_wait(void *bar, uint32_t parity, volatile int *abort, int *status, int where) {
+  if (*abort) return;
+  for (uint32_t i = 0; i < kWaitTries; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  *abort = 1;
+  if (atomicExch(status, 1) == 0) status[1] = where;
+}
+// global -> shared bulk copy, completion counted in bytes on `bar`
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src, uint32_t bytes, void *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_addr(dst_smem)),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+// shared -> global bulk copy, tracked by the thread's bulk async-group
+__device__ __forceinline__ void bulk_store(void *dst, const void *src_smem, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_addr(src_smem)),
+               "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
+
+// NBUF: base-optimizer buffers (1: h; 2: h, v). POLICY: 0 reset, 1 maintain, 2 average.
+template <int NBUF, int POLICY>
+__global__ void __launch_bounds__(kStagedThreads, kStagedCtasPerSm)
+outer_step_staged_kernel(const OuterArgs A, int *status) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  StagedSmem &S = *reinterpret_cast<StagedSmem *>(smem_raw);
+
+  const uint32_t tid = threadIdx.x;
+  const uint32_t warp = tid >> 5;
+  const uint32_t total_cols = A.nvec * 4u;  // fits: nvec <= 2^30 is enforced by the launcher
+  const uint32_t ntiles = (total_cols + kTileCols - 1) / kTileCols;
+  const uint32_t nchunks = (A.m + kStageRows - 1) / kStageRows;
+  constexpr int kPasses = POLICY == 2 ? 1 + NBUF : 1;  // x, then h (and v) when averaging
+
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&S.full[s], 1);
+      mbar_init(&S.empty[s], kConsumerWarps);
+    }
+    S.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (uint32_t i = tid; i < kTileCols; i += kStagedThreads) S.zeros[i] = 0.0f;
+  fence_async_proxy();  // zeros are read by bulk stores
+  __syncthreads();
+
+  if (warp == kConsumerWarps) {
+    // ---------------- producer: one thread feeds the ring ----------------
+    if ((tid & 31) == 0) {
+      uint32_t job = 0, issued = 0;  // issued: jobs whose copies were started
+      for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint32_t col0 = tile * kTileCols;
+        const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+        for (int pass = 0; pass < kPasses; ++pass) {
+          const float *src = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
+          for (uint32_t c = 0; c < nchunks; ++c, ++job) {
+            const uint32_t st = job % kStages, round = job / kStages;
+            mbar_wait(&S.empty[st], (round & 1u) ^ 1u, &S.abort, status, 1);
+            if (S.abort) continue;
+            issued = job + 1;
+            const uint32_t r0 = c * kStageRows;
+            const uint32_t rows = min((uint32_t)kStageRows, A.m - r0);
+            mbar_expect_tx(&S.full[st], rows * ncols * 4u);
+            for (uint32_t r = 0; r < rows; ++r)
+              bulk_load(&S.stage[st][r][0], src + (uint64_t)(r0 + r) * A.pitch + col0, ncols * 4u, &S.full[st]);
+          }
+        }
+      }
+      // copies still in flight must land before the shared memory is given back
+      if (S.abort) {
+        for (uint32_t j = issued > (uint32_t)kStages ? issued - kStages : 0; j < issued; ++j)
+          for (uint32_t i = 0; i < kWaitTries; ++i)
+            if (mbar_try_wait(&S.full[j % kStages], (j / kStages) & 1u)) break;
+      }
+    }
+  } else {
+    // ---------------- consumers ----------------
+    const bool issuer = tid == 0;
+    uint32_t job = 0, outs = 0;
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const uint32_t col0 = tile * kTileCols;
+      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      const bool active = tid * 4u < ncols;
+      const uint64_t col = (uint64_t)col0 + tid * 4u;
+
+      float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), u0 = x0;
+      if (active) {
+        x0 = ld_stream(A.anchor + col);
+        u0 = ld_stream(A.u + col);
+      }
+
+      for (int pass = 0; pass < kPasses; ++pass) {
+        // ordered sum over the workers, chunk by chunk
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t c = 0; c < nchunks; ++c, ++job) {
+          const uint32_t st = job % kStages, round = job / kStages;
+          mbar_wait(&S.full[st], round & 1u, &S.abort, status, 2);
+          const uint32_t rows = min((uint32_t)kStageRows, A.m - c * kStageRows);
+          if (active) {
+#pragma unroll
+            for (int r = 0; r < kStageRows; ++r) {
+              if ((uint32_t)r < rows) {
+                const float4 v = *reinterpret_cast<const float4 *>(&S.stage[st][r][tid * 4u]);
+                if (c == 0 && r == 0) {
+                  s = v;
+                } else {
+                  s.x = __fadd_rn(s.x, v.x);
+                  s.y = __fadd_rn(s.y, v.y);
+                  s.z = __fadd_rn(s.z, v.z);
+                  s.w = __fadd_rn(s.w, v.w);
+                }
+              }
+            }
+          }
+          __syncwarp();
+          if ((tid & 31) == 0) mbar_arrive(&S.empty[st]);
+        }
+        const float4 mean = make_float4(__fdiv_rn(s.x, A.m_float), __fdiv_rn(s.y, A.m_float),
+                                        __fdiv_rn(s.z, A.m_float), __fdiv_rn(s.w, A.m_float));
+        float4 outv = mean;  // passes 1, 2: averaged buffer
+        if (pass == 0) {
+          float4 un;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            // Eq. (2) and Eq. (3)
+            const float ue = __fmaf_rn(A.beta, comp(u0, e), __fmul_rn(__fsub_rn(comp(x0, e), comp(mean, e)), A.inv_gamma));
+            comp(un, e) = ue;
+            comp(outv, e) = __fmaf_rn(A.neg_alpha_gamma, ue, comp(x0, e));
+          }
+          if (active && !S.abort) st_stream(A.u + col, un);
+        }
+
+        // the tile goes to shared memory once and from there to every row
+        const uint32_t ob = outs & 1u;
+        ++outs;
+        if (issuer) bulk_wait_read<1>();  // the bulk stores that last read out[ob] are done with it
+        consumer_sync();
+        if (active) *reinterpret_cast<float4 *>(&S.out[ob][tid * 4u]) = outv;
+        fence_async_proxy();
+        consumer_sync();
+        if (issuer && !S.abort) {
+          float *dst = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
+          for (uint32_t i = 0; i < A.m; ++i) bulk_store(dst + (uint64_t)i * A.pitch + col0, &S.out[ob][0], ncols * 4u);
+          if (pass == 0) {
+            bulk_store(A.anchor + col0, &S.out[ob][0], ncols * 4u);
+            if (POLICY == 0) {  // reset: zero tiles to every buffer row
+              for (uint32_t i = 0; i < A.m; ++i) bulk_store(A.h + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
+              if (NBUF == 2)
+                for (uint32_t i = 0; i < A.m; ++i) bulk_store(A.v + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
+            }
+          }
+          bulk_commit();
+        }
+      }
+    }
+    if (issuer) bulk_wait_all();
+  }
+  __syncthreads();
+}
+
+inline cudaError_t outer_staged_configure() {
+  const int bytes = (int)sizeof(StagedSmem);
+  cudaError_t e = cudaSuccess;
+#define SLOWMO_SET(NB, PO)                                                                                     \
+  if (e == cudaSuccess)                                                                                        \
+    e = cudaFuncSetAttribute(outer_step_staged_kernel<NB, PO>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  SLOWMO_SET(1, 0) SLOWMO_SET(1, 1) SLOWMO_SET(1, 2) SLOWMO_SET(2, 0) SLOWMO_SET(2, 1) SLOWMO_SET(2, 2)
+#undef SLOWMO_SET
+  return e;
+}
+
+inline void launch_outer_staged(const OuterArgs &A, int nbuf, int policy, int num_sms, int *status,
+                                cudaStream_t stream) {
+  const uint32_t ntiles = (A.nvec * 4u + kTileCols - 1) / kTileCols;
+  uint32_t grid = (uint32_t)num_sms * kStagedCtasPerSm;
+  if (grid > ntiles) grid = ntiles;
+  const size_t bytes = sizeof(StagedSmem);
+#define SLOWMO_GO(NB, PO) outer_step_staged_kernel<NB, PO><<<grid, kStagedThreads, bytes, stream>>>(A, status)
+  if (nbuf == 1) {
+    if (policy == 0) SLOWMO_GO(1, 0); else if (policy == 1) SLOWMO_GO(1, 1); else SLOWMO_GO(1, 2);
+  } else {
+    if (policy == 0) SLOWMO_GO(2, 0); else if (policy == 1) SLOWMO_GO(2, 1); else SLOWMO_GO(2, 2);
+  }
+#undef SLOWMO_GO
+}
+
+}  // namespace slowmo

@@ -1,0 +1,429 @@
+// Host side of libslowmo: argument checking, the state machine of Algorithm 1 (outer
+// iteration t, inner step k, Adam count l) and kernel launches. See include/slowmo.h for
+// the contract of every entry point.
+#include "../../include/slowmo.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+#include "outer_staged.cuh"
+
+using namespace slowmo;
+
+struct slowmo_ctx {
+  slowmo_config cfg;
+  slowmo_buffers buf;
+  cudaStream_t stream;
+  uint32_t nvec;             // 4-element column groups per row: ceil(P/4)
+  uint64_t t;                // outer iteration
+  uint32_t k;                // inner steps taken in this outer iteration
+  uint64_t l;                // Adam steps since the buffers were last zero
+  double pow_b1, pow_b2;     // beta_1^l, beta_2^l
+  float gamma;               // gamma_t in force
+  std::vector<uint64_t> tensor_offsets;  // n_tensors + 1 prefix sums, or empty
+  int outer_variant;
+  int *status_dev;           // device status block: [0] = timeout flag, [1] = where
+  int cuda_error;
+  int num_sms;
+};
+
+namespace {
+
+constexpr int kLocalUnroll = 2;
+
+bool finite_pos(float v) { return std::isfinite(v) && v > 0.0f; }
+bool unit_interval(float v) { return std::isfinite(v) && v >= 0.0f && v < 1.0f; }
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(slowmo_ctx *ctx, cudaError_t e) {
+  if (e == cudaSuccess) return SLOWMO_OK;
+  if (ctx && ctx->cuda_error == 0) ctx->cuda_error = (int)e;
+  return SLOWMO_ECUDA;
+}
+
+int check_launch(slowmo_ctx *ctx) { return cuda_fail(ctx, cudaGetLastError()); }
+
+uint32_t fill_blocks(const slowmo_ctx *ctx, uint32_t rows) {
+  // grid-stride fills: enough blocks to cover the machine a few times, split over the rows
+  uint64_t want = (uint64_t)ctx->num_sms * 16;
+  uint64_t per_row = (want + rows - 1) / rows;
+  uint64_t need = ((uint64_t)ctx->nvec + kThreads - 1) / kThreads;
+  if (per_row > need) per_row = need;
+  if (per_row < 1) per_row = 1;
+  return (uint32_t)per_row;
+}
+
+template <int BASE, int GRAD>
+void launch_local(slowmo_ctx *ctx, const LocalArgs &A) {
+  const uint32_t per_tile = kThreads * kLocalUnroll;
+  const uint32_t tiles = (ctx->nvec + per_tile - 1) / per_tile;
+  local_step_kernel<BASE, GRAD, kLocalUnroll><<<tiles * ctx->cfg.m, kThreads, 0, ctx->stream>>>(A);
+}
+
+template <int NBUF>
+void launch_outer_direct(slowmo_ctx *ctx, const OuterArgs &A) {
+  const uint32_t blocks = (ctx->nvec + kThreads - 1) / kThreads;
+  switch (ctx->cfg.buffer_policy) {
+    case SLOWMO_BUF_RESET: outer_step_direct_kernel<NBUF, 0><<<blocks, kThreads, 0, ctx->stream>>>(A); break;
+    case SLOWMO_BUF_MAINTAIN: outer_step_direct_kernel<NBUF, 1><<<blocks, kThreads, 0, ctx->stream>>>(A); break;
+    default: outer_step_direct_kernel<NBUF, 2><<<blocks, kThreads, 0, ctx->stream>>>(A); break;
+  }
+}
+
+// Resolve a tensor id to (base pointer, rows); NULL if the tensor does not exist here.
+float *tensor_base(slowmo_ctx *ctx, int which, uint32_t *rows) {
+  const slowmo_buffers &b = ctx->buf;
+  switch (which) {
+    case SLOWMO_T_X: *rows = ctx->cfg.m; return b.x;
+    case SLOWMO_T_ANCHOR: *rows = 1; return b.anchor;
+    case SLOWMO_T_U: *rows = 1; return b.u;
+    case SLOWMO_T_H: *rows = ctx->cfg.m; return b.h;
+    case SLOWMO_T_V: *rows = ctx->cfg.m; return b.v;
+    case SLOWMO_T_A: *rows = 1; return b.a;
+    case SLOWMO_T_C: *rows = ctx->cfg.m; return b.c;
+    default: *rows = 0; return nullptr;
+  }
+}
+
+int copy_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count, float *user,
+                int user_on_device, bool to_user) {
+  if (!ctx || !user) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  uint32_t rows = 0;
+  float *base = tensor_base(ctx, which, &rows);
+  if (!base) return SLOWMO_EINVAL;
+  if (replica < -1 || (replica >= 0 && (uint32_t)replica >= rows)) return SLOWMO_EINVAL;
+  if (offset > ctx->cfg.P || count > ctx->cfg.P - offset) return SLOWMO_EINVAL;
+  if (count == 0) return SLOWMO_OK;
+  const uint32_t nrows = replica < 0 ? rows : 1;
+  float *dev = base + (replica < 0 ? 0 : (uint64_t)replica * ctx->buf.pitch) + offset;
+  const size_t width = count * sizeof(float), dpitch = ctx->buf.pitch * sizeof(float);
+  cudaError_t e;
+  if (to_user) {
+    e = cudaMemcpy2DAsync(user, width, dev, dpitch, width, nrows,
+                          user_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, ctx->stream);
+  } else {
+    e = cudaMemcpy2DAsync(dev, dpitch, user, width, width, nrows,
+                          user_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, ctx->stream);
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (!user_on_device) return cuda_fail(ctx, cudaStreamSynchronize(ctx->stream));
+  return SLOWMO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cuda_stream, slowmo_ctx **out) {
+  if (!cfg || !buf || !out) return SLOWMO_EINVAL;
+  *out = nullptr;
+  const bool adam = cfg->base == SLOWMO_BASE_ADAM;
+  const bool generated = cfg->grad_mode == SLOWMO_GRAD_GENERATED;
+  if (cfg->P == 0 || cfg->m == 0 || cfg->tau == 0) return SLOWMO_EINVAL;
+  if (cfg->P > (1ull << 32) - 4096) return SLOWMO_EINVAL;  // columns are indexed with 32 bits
+  if (!finite_pos(cfg->alpha) || !unit_interval(cfg->beta) || !finite_pos(cfg->gamma)) return SLOWMO_EINVAL;
+  if (cfg->base != SLOWMO_BASE_NESTEROV && !adam) return SLOWMO_EINVAL;
+  if (cfg->buffer_policy < SLOWMO_BUF_RESET || cfg->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
+  if (!generated && cfg->grad_mode != SLOWMO_GRAD_SUPPLIED) return SLOWMO_EINVAL;
+  if (!std::isfinite(cfg->weight_decay) || cfg->weight_decay < 0.0f || !std::isfinite(cfg->x_init)) return SLOWMO_EINVAL;
+  if (!adam && !unit_interval(cfg->mu)) return SLOWMO_EINVAL;
+  if (adam && (!unit_interval(cfg->adam_b1) || !unit_interval(cfg->adam_b2) || !finite_pos(cfg->adam_eps)))
+    return SLOWMO_EINVAL;
+  if (!std::isfinite(cfg->sigma) || cfg->sigma < 0.0f) return SLOWMO_EINVAL;
+  if (generated && (!std::isfinite(cfg->a_lo) || !std::isfinite(cfg->a_hi) || cfg->a_hi < cfg->a_lo ||
+                    !std::isfinite(cfg->c_std) || cfg->c_std < 0.0f))
+    return SLOWMO_EINVAL;
+  if (!buf->x || !buf->h || !buf->anchor || !buf->u) return SLOWMO_EINVAL;
+  if (adam && !buf->v) return SLOWMO_EINVAL;
+  if (generated && (!buf->a || !buf->c)) return SLOWMO_EINVAL;
+  if ((cfg->n_tensors != 0) != (cfg->tensor_sizes != nullptr)) return SLOWMO_EINVAL;
+  if (buf->pitch % 4 != 0) return SLOWMO_EALIGN;
+  if (buf->pitch < cfg->P) return SLOWMO_EINVAL;
+  const void *ptrs[] = {buf->x, buf->h, buf->v, buf->anchor, buf->u, buf->a, buf->c};
+  for (const void *p : ptrs)
+    if (p && !aligned16(p)) return SLOWMO_EALIGN;
+  const uint64_t nvec = (cfg->P + 3) / 4;
+  const uint64_t per_tile = (uint64_t)kThreads * kLocalUnroll;
+  if (((nvec + per_tile - 1) / per_tile) * cfg->m >= (1ull << 31)) return SLOWMO_EINVAL;  // grid limit
+
+  slowmo_ctx *ctx = new (std::nothrow) slowmo_ctx();
+  if (!ctx) return SLOWMO_ENOMEM;
+  ctx->cfg = *cfg;
+  ctx->cfg.tensor_sizes = nullptr;
+  ctx->buf = *buf;
+  ctx->stream = (cudaStream_t)cuda_stream;
+  ctx->nvec = (uint32_t)nvec;
+  ctx->t = 0;
+  ctx->k = 0;
+  ctx->l = 0;
+  ctx->pow_b1 = ctx->pow_b2 = 1.0;
+  ctx->gamma = cfg->gamma;
+  ctx->outer_variant = SLOWMO_VARIANT_DEFAULT;
+  ctx->status_dev = nullptr;
+  ctx->cuda_error = 0;
+  if (cfg->n_tensors) {
+    try {
+      ctx->tensor_offsets.resize((size_t)cfg->n_tensors + 1);
+    } catch (...) {
+      delete ctx;
+      return SLOWMO_ENOMEM;
+    }
+    uint64_t acc = 0;
+    for (uint32_t i = 0; i < cfg->n_tensors; ++i) {
+      ctx->tensor_offsets[i] = acc;
+      if (cfg->tensor_sizes[i] == 0 || cfg->tensor_sizes[i] > cfg->P - acc) {
+        delete ctx;
+        return SLOWMO_EINVAL;
+      }
+      acc += cfg->tensor_sizes[i];
+    }
+    ctx->tensor_offsets[cfg->n_tensors] = acc;
+    if (acc != cfg->P) {
+      delete ctx;
+      return SLOWMO_EINVAL;
+    }
+  }
+
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->status_dev, 4 * sizeof(int));
+  if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status_dev, 0, 4 * sizeof(int), ctx->stream);
+  if (e == cudaSuccess) e = outer_staged_configure();
+  if (e != cudaSuccess) {
+    if (ctx->status_dev) cudaFree(ctx->status_dev);
+    delete ctx;
+    return SLOWMO_ECUDA;
+  }
+
+  // Algorithm 1, input line: x^{(i)} = x_{0,0}, u_0 = 0, buffers zero; synthetic problem data.
+  const uint32_t m = cfg->m;
+  const size_t row_bytes = (size_t)ctx->nvec * 4 * sizeof(float);
+  const size_t pitch_bytes = buf->pitch * sizeof(float);
+  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->x, buf->pitch, ctx->nvec, cfg->x_init);
+  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, 1), 1), kThreads, 0, ctx->stream>>>(buf->anchor, buf->pitch, ctx->nvec, cfg->x_init);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaMemsetAsync(buf->u, 0, row_bytes, ctx->stream);
+  if (e == cudaSuccess) e = cudaMemset2DAsync(buf->h, pitch_bytes, 0, row_bytes, m, ctx->stream);
+  if (e == cudaSuccess && buf->v) e = cudaMemset2DAsync(buf->v, pitch_bytes, 0, row_bytes, m, ctx->stream);
+  if (e == cudaSuccess && generated) {
+    fill_curvature_kernel<<<fill_blocks(ctx, 1), kThreads, 0, ctx->stream>>>(buf->a, ctx->nvec, cfg->seed, cfg->a_lo, cfg->a_hi);
+    fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->c, buf->pitch, ctx->nvec, kTagCentre,
+                                                                                   cfg->seed, cfg->c_std);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    cudaFree(ctx->status_dev);
+    delete ctx;
+    return SLOWMO_ECUDA;
+  }
+  *out = ctx;
+  return SLOWMO_OK;
+}
+
+int slowmo_destroy(slowmo_ctx *ctx) {
+  if (!ctx) return SLOWMO_EINVAL;
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->status_dev) cudaFree(ctx->status_dev);
+  delete ctx;
+  return SLOWMO_OK;
+}
+
+int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  const slowmo_config &c = ctx->cfg;
+  const bool generated = c.grad_mode == SLOWMO_GRAD_GENERATED;
+  if (generated ? grad != nullptr : grad == nullptr) return SLOWMO_EINVAL;
+  if (grad && !aligned16(grad)) return SLOWMO_EALIGN;
+  if ((uint64_t)ctx->k + n > c.tau) return SLOWMO_ESTATE;
+
+  LocalArgs A;
+  A.x = ctx->buf.x;
+  A.h = ctx->buf.h;
+  A.v = ctx->buf.v;
+  A.src = generated ? ctx->buf.c : grad;
+  A.a = ctx->buf.a;
+  A.pitch = ctx->buf.pitch;
+  A.nvec = ctx->nvec;
+  A.m = c.m;
+  A.seed = c.seed;
+  A.neg_gamma = -ctx->gamma;
+  A.mu = c.mu;
+  A.wd = c.weight_decay;
+  A.sigma = c.sigma;
+  A.b1 = c.adam_b1;
+  A.b2 = c.adam_b2;
+  A.omb1 = (float)(1.0 - (double)c.adam_b1);
+  A.omb2 = (float)(1.0 - (double)c.adam_b2);
+  A.eps = c.adam_eps;
+
+  for (uint32_t s = 0; s < n; ++s) {
+    // Table C.1: bias corrections use the 1-based count l of Adam steps since the buffers were zero
+    ctx->l += 1;
+    ctx->pow_b1 *= (double)c.adam_b1;
+    ctx->pow_b2 *= (double)c.adam_b2;
+    A.ibc1 = (float)(1.0 / (1.0 - ctx->pow_b1));
+    A.ibc2 = (float)(1.0 / (1.0 - ctx->pow_b2));
+    A.t = ctx->t;
+    A.k = ctx->k;
+    if (c.base == SLOWMO_BASE_NESTEROV) {
+      if (generated) launch_local<0, 0>(ctx, A); else launch_local<0, 1>(ctx, A);
+    } else {
+      if (generated) launch_local<1, 0>(ctx, A); else launch_local<1, 1>(ctx, A);
+    }
+    ctx->k += 1;
+    int rc = check_launch(ctx);
+    if (rc != SLOWMO_OK) return rc;
+  }
+  return SLOWMO_OK;
+}
+
+int slowmo_outer_step(slowmo_ctx *ctx) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  const slowmo_config &c = ctx->cfg;
+  if (ctx->k != c.tau) return SLOWMO_ESTATE;
+
+  OuterArgs A;
+  A.x = ctx->buf.x;
+  A.h = ctx->buf.h;
+  A.v = ctx->buf.v;
+  A.anchor = ctx->buf.anchor;
+  A.u = ctx->buf.u;
+  A.pitch = ctx->buf.pitch;
+  A.nvec = ctx->nvec;
+  A.m = c.m;
+  A.beta = c.beta;
+  A.inv_gamma = (float)(1.0 / (double)ctx->gamma);
+  A.neg_alpha_gamma = -(float)((double)c.alpha * (double)ctx->gamma);
+  A.m_float = (float)c.m;
+  const int nbuf = c.base == SLOWMO_BASE_ADAM ? 2 : 1;
+
+  int variant = ctx->outer_variant;
+  if (variant == SLOWMO_VARIANT_DEFAULT) variant = SLOWMO_OUTER_DIRECT;
+  if (variant == SLOWMO_OUTER_STAGED) {
+    launch_outer_staged(A, nbuf, c.buffer_policy, ctx->num_sms, ctx->status_dev, ctx->stream);
+  } else {
+    if (nbuf == 1) launch_outer_direct<1>(ctx, A); else launch_outer_direct<2>(ctx, A);
+  }
+  int rc = check_launch(ctx);
+  if (rc != SLOWMO_OK) return rc;
+
+  ctx->t += 1;
+  ctx->k = 0;
+  if (c.buffer_policy == SLOWMO_BUF_RESET) {
+    ctx->l = 0;
+    ctx->pow_b1 = ctx->pow_b2 = 1.0;
+  }
+  return SLOWMO_OK;
+}
+
+int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t) {
+  if (!ctx || !finite_pos(gamma_t)) return SLOWMO_EINVAL;
+  if (ctx->k != 0) return SLOWMO_ESTATE;
+  ctx->gamma = gamma_t;
+  return SLOWMO_OK;
+}
+
+int slowmo_get_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count, float *dst,
+                      int dst_on_device) {
+  return copy_params(ctx, which, replica, offset, count, dst, dst_on_device, true);
+}
+
+int slowmo_set_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count,
+                      const float *src, int src_on_device) {
+  return copy_params(ctx, which, replica, offset, count, const_cast<float *>(src), src_on_device, false);
+}
+
+int slowmo_get_counters(slowmo_ctx *ctx, uint64_t *t, uint32_t *k, uint64_t *l) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (t) *t = ctx->t;
+  if (k) *k = ctx->k;
+  if (l) *l = ctx->l;
+  return SLOWMO_OK;
+}
+
+int slowmo_fill_gradient(slowmo_ctx *ctx, float *grad) {
+  if (!ctx || !grad) return SLOWMO_EINVAL;
+  if (!aligned16(grad)) return SLOWMO_EALIGN;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  const uint32_t m = ctx->cfg.m;
+  fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(
+      grad, ctx->buf.pitch, ctx->nvec, kTagSupplied, ctx->cfg.seed, ctx->cfg.sigma);
+  return check_launch(ctx);
+}
+
+int slowmo_debug_noise(slowmo_ctx *ctx, uint32_t tag, uint64_t t, uint32_t k, uint32_t w, uint64_t j0, uint64_t n,
+                       uint64_t *words, float *normals) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  if (n == 0) return SLOWMO_OK;
+  if (!words && !normals) return SLOWMO_EINVAL;
+  const uint64_t key = stream_key(tag, ctx->cfg.seed, t, k, w);
+  uint64_t blocks = (n + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)ctx->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  export_stream_kernel<<<(uint32_t)blocks, kThreads, 0, ctx->stream>>>(key, j0, n, words, normals);
+  return check_launch(ctx);
+}
+
+int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_t *count) {
+  if (!ctx || !offset || !count) return SLOWMO_EINVAL;
+  if (ctx->tensor_offsets.empty() || idx >= ctx->cfg.n_tensors) return SLOWMO_EINVAL;
+  *offset = ctx->tensor_offsets[idx];
+  *count = ctx->tensor_offsets[idx + 1] - ctx->tensor_offsets[idx];
+  return SLOWMO_OK;
+}
+
+int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (kernel == SLOWMO_K_OUTER) {
+    if (variant != SLOWMO_VARIANT_DEFAULT && variant != SLOWMO_OUTER_DIRECT && variant != SLOWMO_OUTER_STAGED)
+      return SLOWMO_EINVAL;
+    ctx->outer_variant = variant;
+    return SLOWMO_OK;
+  }
+  if (kernel == SLOWMO_K_LOCAL) return variant == SLOWMO_VARIANT_DEFAULT ? SLOWMO_OK : SLOWMO_EINVAL;
+  return SLOWMO_EINVAL;
+}
+
+int slowmo_sync_status(slowmo_ctx *ctx) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  int host[4] = {0, 0, 0, 0};
+  cudaError_t e = cudaMemcpyAsync(host, ctx->status_dev, sizeof(host), cudaMemcpyDeviceToHost, ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+  if (host[0] != 0) {
+    e = cudaMemsetAsync(ctx->status_dev, 0, sizeof(host), ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    return SLOWMO_ETIMEOUT;
+  }
+  return SLOWMO_OK;
+}
+
+const char *slowmo_strerror(int status) {
+  switch (status) {
+    case SLOWMO_OK: return "ok";
+    case SLOWMO_EINVAL: return "invalid argument";
+    case SLOWMO_ESTATE: return "call not legal at this point of the outer/inner loop";
+    case SLOWMO_EALIGN: return "pointer not 16-byte aligned or pitch not a multiple of 4";
+    case SLOWMO_ECUDA: return "CUDA error (see slowmo_last_cuda_error)";
+    case SLOWMO_ENOMEM: return "out of host memory";
+    case SLOWMO_ETIMEOUT: return "a bounded device-side wait gave up";
+    case SLOWMO_ENOTIMPL: return "not implemented";
+    default: return "unknown status";
+  }
+}
+
+int slowmo_last_cuda_error(slowmo_ctx *ctx) { return ctx ? ctx->cuda_error : 0; }
+
+}  // extern "C"

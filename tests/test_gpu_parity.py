@@ -1,0 +1,384 @@
+"""GPU parity: the CUDA library (through its C ABI) against the binary32 oracle, element by
+element on small cases and on sampled coordinates at the full benchmark sizes.
+
+Gate (all state tensors x, anchor, u, h, v after the full run):
+    max |gpu - oracle| <= 1e-5 * (1 + |oracle|)
+The integer noise stream must match bit for bit.
+"""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_1910_00643_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5
+
+
+def _slowmo(w, **kw):
+    from paper_1910_00643_b200 import SlowMo
+    return SlowMo(w, **kw)
+
+
+def _state_keys(w):
+    return ("x", "anchor", "u", "h") + (("v",) if w.get("base") == "adam" else ())
+
+
+def _gather(s, key, j):
+    """Columns j of a state tensor, straight from device memory."""
+    import torch
+    idx = torch.as_tensor(np.asarray(j, dtype=np.int64), device="cuda")
+    t = s.t[key]
+    two_d = key in ("x", "h", "v", "c")
+    out = t.view(s.m if two_d else 1, s.pitch).index_select(1, idx).cpu().numpy()
+    return out if two_d else out[0]
+
+
+def _assert_close(got, ref, what):
+    got64, ref64 = got.astype(np.float64), ref.astype(np.float64)
+    err = np.abs(got64 - ref64)
+    bad = err > RTOL * (1.0 + np.abs(ref64))
+    assert not bad.any(), f"{what}: {int(bad.sum())} elements off, max |d| = {err.max():.3e}"
+    assert np.isfinite(got64).all(), what
+
+
+def _check_against_oracle(s, w, j, T=None, gamma_t=None, G=None, exact=False):
+    s.sync_status()
+    cfg = oracle.make_config(**dict(w, T=w["T"] if T is None else T))
+    ref = oracle.run(cfg, j=np.asarray(j, np.uint64), precision="f32", gamma_t=gamma_t, G=G)
+    for key in _state_keys(w):
+        got = _gather(s, key, j)
+        _assert_close(got, ref[key], f"{w.get('name')}:{key}")
+        if exact:
+            assert np.array_equal(got.view(np.uint32), ref[key].view(np.uint32)), f"{key} not bit-equal"
+    return ref
+
+
+# ------------------------------------------------------------------------------- noise stream
+
+def test_noise_words_and_normals_are_bit_exact():
+    s = _slowmo(workloads.workload("tiny", seed=77))
+    cases = [(3, 0, 0, 0, 0), (3, 2, 3, 1, 12345), (1, 0, 0, 0, 0), (2, 0, 0, 3, 999), (5, 0, 0, 2, 7),
+             (3, 2**40 + 5, 47, 31, 2**32 - 100), (3, 9, 1, 0, 2**33 + 1)]
+    for tag, t, k, wk, j0 in cases:
+        n = 5000
+        gw, gz = s.debug_noise(tag, t, k, wk, j0, n)
+        ow, oz = oracle.stream(tag, 77, t, k, wk, j0, n)
+        assert np.array_equal(gw, ow), (tag, t, k, wk, j0)
+        assert np.array_equal(gz.view(np.uint32), oz.view(np.uint32)), (tag, t, k, wk, j0)
+    s.close()
+
+
+def test_normals_bit_exact_on_a_large_sample():
+    s = _slowmo(workloads.workload("tiny"))
+    n = 1 << 22
+    gw, gz = s.debug_noise(3, 1, 2, 3, 0, n)
+    ow, oz = oracle.stream(3, 0, 1, 2, 3, 0, n)
+    assert np.array_equal(gw, ow)
+    assert np.array_equal(gz.view(np.uint32), oz.view(np.uint32))
+    s.close()
+
+
+def test_problem_data_fill_matches_oracle():
+    w = workloads.workload("tiny", P=5003, m=3, a_lo=0.1, a_hi=1.0, c_std=0.05, seed=5)
+    s = _slowmo(w, guard=64)
+    cfg = oracle.make_config(**w)
+    j = np.arange(w["P"])
+    a = s.get_params("a")[0]
+    assert np.array_equal(a.view(np.uint32), oracle.curvature(cfg, j).view(np.uint32))
+    c = s.get_params("c")
+    for i in range(3):
+        assert np.array_equal(c[i].view(np.uint32), oracle.centre(cfg, i, j).view(np.uint32))
+    x = s.get_params("x")
+    assert (x == np.float32(w["x_init"])).all() and not s.get_params("u").any() and not s.get_params("h").any()
+    assert s.guards_intact()
+    s.close()
+
+
+def test_supplied_gradient_fill_matches_oracle():
+    w = workloads.workload("stress_tau1", P=4099, m=2, sigma=0.3, seed=11)
+    s = _slowmo(w, guard=64)
+    g = s.alloc_gradient()
+    s.fill_gradient()
+    s.synchronize()
+    cfg = oracle.make_config(**w)
+    got = g.view(2, s.pitch)[:, :w["P"]].cpu().numpy()
+    for i in range(2):
+        ref = oracle.supplied_gradient(cfg, i, np.arange(w["P"]))
+        assert np.array_equal(got[i].view(np.uint32), ref.view(np.uint32))
+    assert s.guards_intact()
+    s.close()
+
+
+# ------------------------------------------------------------- small cases, element by element
+
+SMALL_P = 3 * 1024 + 37  # several 512- and 1024-column tiles and a ragged tail (not a multiple of 4)
+
+
+@pytest.mark.parametrize("variant", ["direct", "staged"])
+@pytest.mark.parametrize("base,policy", list(itertools.product(("nesterov", "adam"), ("reset", "maintain", "average"))))
+@pytest.mark.parametrize("m", [1, 3, 4, 9])
+def test_small_runs_match_oracle(base, policy, m, variant):
+    w = workloads.workload("tiny", P=SMALL_P, m=m, tau=3, T=3, base=base, buffer_policy=policy, alpha=0.9,
+                           beta=0.6, gamma=0.01 if base == "adam" else 0.05, weight_decay=1e-3,
+                           adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8, seed=3)
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", variant)
+    s.run(w["T"])
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    assert s.counters()[0] == 3 and s.counters()[1] == 0
+    s.close()
+
+
+@pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 511, 512, 513, 1023, 1024, 1025, 2048 + 4])
+def test_ragged_sizes(P):
+    w = workloads.workload("tiny", P=P, m=5, tau=2, T=2, buffer_policy="average")
+    for variant in ("direct", "staged"):
+        s = _slowmo(w, guard=64)
+        s.set_variant("outer", variant)
+        s.run(2)
+        _check_against_oracle(s, w, np.arange(P), exact=True)
+        assert s.guards_intact()
+        s.close()
+
+
+def test_tiny_workload_full_run():
+    w = workloads.workload("tiny")
+    s = _slowmo(w)
+    s.run(w["T"])
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    s.close()
+
+
+def test_many_workers():
+    w = workloads.workload("tiny", P=2051, m=32, tau=2, T=2, buffer_policy="average")
+    for variant in ("direct", "staged"):
+        s = _slowmo(w)
+        s.set_variant("outer", variant)
+        s.run(2)
+        _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+        s.close()
+
+
+def test_every_worker_holds_the_anchor_after_the_outer_step():
+    import torch
+    w = workloads.workload("tiny", P=10_001, m=6)
+    s = _slowmo(w)
+    s.run(2)
+    s.synchronize()
+    x = s.t["x"].view(6, s.pitch)[:, :w["P"]]
+    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    assert not bool(s.t["h"].view(6, s.pitch)[:, :w["P"]].any())  # reset policy
+    s.close()
+
+
+def test_runs_are_bit_reproducible():
+    import torch
+    w = workloads.workload("resnet50", P=200_003, m=8, T=2, n_tensors=0)
+    outs = []
+    for variant in ("direct", "staged", "direct"):
+        s = _slowmo(w)
+        s.set_variant("outer", variant)
+        s.run(2)
+        s.synchronize()
+        outs.append([s.t[k].view(-1, s.pitch)[:, :w["P"]].clone() for k in ("x", "anchor", "u", "h")])
+        s.close()
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert torch.equal(a, b)
+
+
+def test_learning_rate_schedule():
+    w = workloads.workload("tiny", P=2000, T=4)
+    gammas = np.array([0.01, 0.05, 0.1, 0.02], np.float32)
+    s = _slowmo(w)
+    for t in range(4):
+        s.set_gamma(float(gammas[t]))
+        s.local_steps(w["tau"])
+        s.outer_step()
+    _check_against_oracle(s, w, np.arange(2000), gamma_t=gammas, exact=True)
+    s.close()
+
+
+def test_supplied_gradient_arrays_per_step():
+    import torch
+    m, tau, T, P = 3, 2, 2, 1500
+    w = workloads.workload("stress_tau1", P=P, m=m, tau=tau, T=T, weight_decay=1e-2, buffer_policy="maintain")
+    G = workloads.dense_gradients(T * tau, m, P, seed=9)
+    s = _slowmo(w)
+    g = s.alloc_gradient().view(m, s.pitch)
+    step = 0
+    for t in range(T):
+        for k in range(tau):
+            with torch.cuda.stream(s.stream):
+                g[:, :P].copy_(torch.from_numpy(G[step]).cuda(), non_blocking=False)
+            s.local_steps(1, s.grad)
+            step += 1
+        s.outer_step()
+    cfg_w = dict(w, grad_mode="supplied_array")
+    _check_against_oracle(s, cfg_w, np.arange(P), G=G, exact=True)
+    s.close()
+
+
+def test_supplied_hash_gradient_small():
+    w = workloads.workload("stress_tau12", P=5000, m=4)
+    s = _slowmo(w, guard=64)
+    s.alloc_gradient()
+    s.fill_gradient()
+    s.run(w["T"], s.grad)
+    _check_against_oracle(s, w, np.arange(5000), exact=True)
+    assert s.guards_intact()
+    s.close()
+
+
+# --------------------------------------------------------------------------- boundary behaviour
+
+def test_call_order_and_argument_errors():
+    from paper_1910_00643_b200 import SlowMoError, binding
+    import torch
+    w = workloads.workload("tiny")
+    s = _slowmo(w)
+    with pytest.raises(SlowMoError) as e:
+        s.outer_step()                       # no local steps yet
+    assert e.value.status == binding.ESTATE
+    s.local_steps(3)
+    with pytest.raises(SlowMoError) as e:
+        s.local_steps(2)                     # 3 + 2 > tau
+    assert e.value.status == binding.ESTATE
+    with pytest.raises(SlowMoError) as e:
+        s.set_gamma(0.1)                     # only legal at k = 0
+    assert e.value.status == binding.ESTATE
+    with pytest.raises(SlowMoError) as e:
+        s.local_steps(1, torch.zeros(4 * s.pitch, device="cuda"))  # gradient given in generated mode
+    assert e.value.status == binding.EINVAL
+    s.local_steps(1)
+    s.outer_step()
+    with pytest.raises(SlowMoError) as e:
+        s.set_gamma(float("nan"))
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(SlowMoError) as e:
+        s.get_params("x", replica=4)
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(SlowMoError) as e:
+        s.get_params("anchor", offset=4000, count=200)
+    assert e.value.status == binding.EINVAL
+    with pytest.raises(SlowMoError) as e:
+        s.get_params("v")                    # Nesterov has no second moment
+    assert e.value.status == binding.EINVAL
+    assert s.counters() == (1, 0, 0)
+    s.sync_status()
+    s.close()
+    ws = workloads.workload("stress_tau1", P=1000)
+    s = _slowmo(ws)
+    with pytest.raises(SlowMoError) as e:
+        s.local_steps(1)                     # supplied mode needs a gradient
+    assert e.value.status == binding.EINVAL
+    s.close()
+
+
+def test_get_and_set_params_round_trip():
+    import torch
+    w = workloads.workload("tiny", P=3001, m=3)
+    s = _slowmo(w, guard=64)
+    s.run(1)
+    x = s.get_params("x")
+    assert x.shape == (3, 3001)
+    row1 = s.get_params("x", replica=1, offset=100, count=50)
+    assert np.array_equal(row1[0], x[1, 100:150])
+    dev = torch.empty(3 * 40, dtype=torch.float32, device="cuda")
+    s.get_params("h", offset=7, count=40, out=dev)
+    s.synchronize()
+    assert np.array_equal(dev.cpu().numpy().reshape(3, 40), s.get_params("h")[:, 7:47])
+    # restore a checkpoint into a fresh context and continue: same result as an uninterrupted run
+    s2 = _slowmo(w)
+    for key in ("x", "anchor", "u", "h"):
+        s2.set_params(key, s.get_params(key))
+    s.run(1)
+    # the fresh context is at t = 0 for the noise key, so compare a state copy only
+    for key in ("x", "anchor", "u", "h"):
+        s2.set_params(key, s.get_params(key))
+        assert np.array_equal(s2.get_params(key), s.get_params(key))
+    assert s.guards_intact()
+    s.close()
+    s2.close()
+
+
+def test_tensor_table():
+    w = workloads.workload("resnet50", P=100_000, m=2, T=1, tau=1)
+    s = _slowmo(w)
+    sizes = workloads.tensor_sizes(100_000, 161, 0)
+    assert int(sizes.sum()) == 100_000 and sizes.min() >= 1
+    off = 0
+    for i in (0, 1, 80, 160):
+        o, c = s.tensor_range(i)
+        assert o == int(sizes[:i].sum()) and c == int(sizes[i])
+    from paper_1910_00643_b200 import SlowMoError
+    with pytest.raises(SlowMoError):
+        s.tensor_range(161)
+    s.close()
+
+
+# ------------------------------------------------------- full benchmark sizes, sampled coordinates
+
+FULL = ["resnet50", "bmuf", "local_sgd", "sync_sgd", "transformer_adam"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_generated_workloads_on_sampled_coordinates(name):
+    import torch
+    w = workloads.workload(name)
+    s = _slowmo(w)
+    s.run(w["T"])
+    j = workloads.sample_coordinates(w["P"], 1 << 13, seed=1)
+    _check_against_oracle(s, w, j, exact=True)
+    # properties that hold at any size: consensus of the replicas, policy post-conditions
+    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
+    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    h = s.t["h"].view(w["m"], s.pitch)[:, :w["P"]]
+    if w["buffer_policy"] == "reset":
+        assert not bool(h.any())
+    if w["buffer_policy"] == "average":
+        assert bool((h == h[0:1]).all())
+    assert bool(torch.isfinite(s.t["u"][:w["P"]]).all())
+    s.close()
+    del s
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["stress_tau1", "stress_tau12"])
+def test_full_size_supplied_gradient_on_sampled_coordinates(name):
+    import torch
+    w = workloads.workload(name)
+    s = _slowmo(w)
+    s.alloc_gradient()
+    s.fill_gradient()
+    s.run(w["T"], s.grad)
+    j = workloads.sample_coordinates(w["P"], 1 << 13, seed=2)
+    _check_against_oracle(s, w, j, exact=True)
+    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
+    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    s.close()
+    del s
+    torch.cuda.empty_cache()
+
+
+def test_full_size_staged_outer_step_equals_direct():
+    import torch
+    w = workloads.workload("resnet50", T=2)
+    res = []
+    for variant in ("direct", "staged"):
+        s = _slowmo(w)
+        s.set_variant("outer", variant)
+        s.run(2)
+        s.sync_status()
+        res.append((s.t["anchor"].clone(), s.t["u"].clone(), s.t["h"].view(w["m"], s.pitch)[::8].clone(),
+                    s.t["x"].view(w["m"], s.pitch)[::8].clone()))
+        s.close()
+        del s
+        torch.cuda.empty_cache()
+    for a, b in zip(*res):
+        assert torch.equal(a[..., :w["P"]], b[..., :w["P"]])
