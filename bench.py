@@ -263,6 +263,17 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
 
 # -------------------------------------------------------------------------------------- arms
 
+def size_overrides(args):
+    """Optional smaller problem (for profiler captures); the default is the named workload."""
+    over = {}
+    for key in ("P", "m", "tau"):
+        if getattr(args, key) is not None:
+            over[key] = getattr(args, key)
+    if "P" in over:
+        over["n_tensors"] = 0
+    return over
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -276,7 +287,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
 
-    w = workloads.workload(args.workload)
+    w = workloads.workload(args.workload, **size_overrides(args))
     peak, peak_kind = measured_peak()
     s = SlowMo(w)
     if args.outer_variant:
@@ -295,7 +306,7 @@ def run_ours(args):
 
     # end to end: host buffers in and out through the C ABI
     e2e = None
-    if w["grad_mode"] == "generated":
+    if w["grad_mode"] == "generated" and not args.no_e2e:
         host_in = torch.empty((w["m"], w["P"]), dtype=torch.float32, pin_memory=True)
         host_out = torch.empty((1, w["P"]), dtype=torch.float32, pin_memory=True)
         s.get_params("c", out=host_in)  # the same per-worker data the device-resident run used
@@ -381,6 +392,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50")
     ap.add_argument("--outer-variant", default=None, choices=[None, "direct", "staged"])
+    ap.add_argument("--P", type=int, default=None, help="override the workload's parameter count")
+    ap.add_argument("--m", type=int, default=None, help="override the workload's worker count")
+    ap.add_argument("--tau", type=int, default=None, help="override the workload's inner steps")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--no-stress", action="store_true", help="skip the P=1e9 per-kernel measurement")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)

@@ -44,8 +44,10 @@ def lib():
         L.oracle_stream_key.argtypes = [C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint32]
         L.oracle_word_to_unit.restype = C.c_float
         L.oracle_word_to_unit.argtypes = [C.c_uint64]
-        L.oracle_word_to_normal.restype = C.c_float
-        L.oracle_word_to_normal.argtypes = [C.c_uint64]
+        L.oracle_word_to_normal_pair.restype = None
+        L.oracle_word_to_normal_pair.argtypes = [C.c_uint64, C.POINTER(C.c_float * 2)]
+        L.oracle_stream_normal.restype = C.c_float
+        L.oracle_stream_normal.argtypes = [C.c_uint64, C.c_uint64]
         L.oracle_stream_export.restype = None
         L.oracle_stream_export.argtypes = [C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint32,
                                            C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p]
@@ -112,8 +114,16 @@ def run(cfg, *, j=None, j0=0, n=None, precision="f32", gamma_t=None, G=None, wan
     return out
 
 
+def normal_pair(word):
+    """The two Box-Muller normals (cosine, sine) made from one 64-bit word."""
+    z = (C.c_float * 2)()
+    lib().oracle_word_to_normal_pair(word, C.byref(z))
+    return float(z[0]), float(z[1])
+
+
 def stream(tag, seed, t, k, w, j0, n, words=True, normals=True):
-    """Words (uint64) and/or binary32 normals of one noise stream for j0 <= j < j0+n."""
+    """For j0 <= j < j0+n: words j of the stream (uint64) and/or the binary32 normals of
+    coordinates j (coordinate j uses output j & 1 of the pair made from word j >> 1)."""
     wd = np.empty(n, np.uint64) if words else None
     z = np.empty(n, np.float32) if normals else None
     lib().oracle_stream_export(tag, seed, t, k, w, j0, n, _ptr(wd), _ptr(z))

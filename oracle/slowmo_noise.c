@@ -5,7 +5,8 @@
  *
  * The paper (Eq. 1) only assumes a stochastic gradient oracle per worker; the concrete
  * stream below is this project's stand-in for it: a SplitMix64 hash of
- * (seed, outer t, local k, worker w, coordinate j) mapped to N(0,1) by Box-Muller.
+ * (seed, outer t, local k, worker w, coordinate j) mapped to N(0,1) by Box-Muller, both
+ * outputs of each Box-Muller pair being used (for coordinates 2q and 2q+1).
  *
  * Built with -ffp-contract=off: every rounding below is written out; fused operations
  * are explicit fmaf calls.
@@ -80,11 +81,11 @@ static float ln_unit24(uint32_t n) {
 }
 
 /*
- * cos(2 pi k2 / 2^24) for a 24-bit integer k2, in binary32.
+ * cos and sin of the angle 2 pi k2 / 2^24 for a 24-bit integer k2, in binary32.
  * The top two bits pick the quadrant; inside the quadrant the angle psi = (pi/2) r / 2^22
  * is reflected about pi/4 so that a Taylor polynomial is only ever evaluated on [0, pi/4].
  */
-static float cos_turn24(uint32_t k2) {
+static void cos_sin_turn24(uint32_t k2, float *cos_out, float *sin_out) {
   uint32_t q = k2 >> 22;
   uint32_t r = k2 & 0x3FFFFFu;
   int reflected = r > 0x200000u;
@@ -114,32 +115,45 @@ static float cos_turn24(uint32_t k2) {
   /* cos psi and sin psi of the un-reflected in-quadrant angle */
   float cos_psi = reflected ? sin_t : cos_t;
   float sin_psi = reflected ? cos_t : sin_t;
-  switch (q) { /* cos(q pi/2 + psi) */
-    case 0: return cos_psi;
-    case 1: return -sin_psi;
-    case 2: return -cos_psi;
-    default: return sin_psi;
+  switch (q) { /* angle = q pi/2 + psi */
+    case 0: *cos_out = cos_psi;  *sin_out = sin_psi;  break;
+    case 1: *cos_out = -sin_psi; *sin_out = cos_psi;  break;
+    case 2: *cos_out = -cos_psi; *sin_out = -sin_psi; break;
+    default: *cos_out = sin_psi; *sin_out = -cos_psi; break;
   }
 }
 
 /*
- * Box-Muller, cosine branch: z = sqrt(-2 ln u1) cos(2 pi u2), with
- * u1 = (k1+1) 2^-24 in (0,1] from bits 63..40 and u2 = k2 2^-24 in [0,1) from bits 39..16.
+ * Box-Muller: one word gives the two independent normals
+ *   z[0] = sqrt(-2 ln u1) cos(2 pi u2),  z[1] = sqrt(-2 ln u1) sin(2 pi u2),
+ * with u1 = (k1+1) 2^-24 in (0,1] from bits 63..40 and u2 = k2 2^-24 in [0,1) from bits 39..16.
  */
-float oracle_word_to_normal(uint64_t r) {
+void oracle_word_to_normal_pair(uint64_t r, float z[2]) {
   uint32_t k1 = (uint32_t)(r >> 40);
   uint32_t k2 = (uint32_t)(r >> 16) & 0xFFFFFFu;
   float radius = sqrtf(-2.0f * ln_unit24(k1 + 1));
-  return radius * cos_turn24(k2);
+  float c, s;
+  cos_sin_turn24(k2, &c, &s);
+  z[0] = radius * c;
+  z[1] = radius * s;
+}
+
+/*
+ * The normal of coordinate j in the stream `key`: coordinates 2q and 2q+1 share word q of
+ * the stream and take the cosine and the sine output of its Box-Muller pair.
+ */
+float oracle_stream_normal(uint64_t key, uint64_t j) {
+  float z[2];
+  oracle_word_to_normal_pair(oracle_stream_word(key, j >> 1), z);
+  return z[j & 1];
 }
 
 void oracle_stream_export(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, uint32_t w,
                           uint64_t j0, uint64_t n, uint64_t *words, float *normals) {
   uint64_t key = oracle_stream_key(tag, seed, t, k, w);
   for (uint64_t i = 0; i < n; ++i) {
-    uint64_t r = oracle_stream_word(key, j0 + i);
-    if (words) words[i] = r;
-    if (normals) normals[i] = oracle_word_to_normal(r);
+    if (words) words[i] = oracle_stream_word(key, j0 + i);
+    if (normals) normals[i] = oracle_stream_normal(key, j0 + i);
   }
 }
 
@@ -153,11 +167,11 @@ float oracle_curvature(const oracle_config *cfg, uint64_t j) {
 /* c_{w,j} = c_std z, z from worker w's centre stream. */
 float oracle_centre(const oracle_config *cfg, uint32_t w, uint64_t j) {
   uint64_t key = oracle_stream_key(ORACLE_TAG_CENTRE, cfg->seed, 0, 0, w);
-  return cfg->c_std * oracle_word_to_normal(oracle_stream_word(key, j));
+  return cfg->c_std * oracle_stream_normal(key, j);
 }
 
 /* G_{w,j} = sigma z, z from worker w's supplied-gradient stream. */
 float oracle_supplied_gradient(const oracle_config *cfg, uint32_t w, uint64_t j) {
   uint64_t key = oracle_stream_key(ORACLE_TAG_SUPPLIED, cfg->seed, 0, 0, w);
-  return cfg->sigma * oracle_word_to_normal(oracle_stream_word(key, j));
+  return cfg->sigma * oracle_stream_normal(key, j);
 }

@@ -44,7 +44,7 @@ static real gradient(const oracle_config *cfg, uint32_t i, uint64_t j, uint32_t 
   if (cfg->grad_mode == ORACLE_GRAD_GENERATED) {
     /* F_i(x) = 1/2 sum_j a_j (x_j - c_{i,j})^2, gradient a_j (x_j - c_{i,j}), plus sigma z */
     uint64_t key = oracle_stream_key(ORACLE_TAG_GRADNOISE, cfg->seed, t, k, i);
-    real z = (real)oracle_word_to_normal(oracle_stream_word(key, j));
+    real z = (real)oracle_stream_normal(key, j);
     real noise = (real)cfg->sigma * z;
     real e = x - c_ij;
     g = FMA(a_j, e, noise);

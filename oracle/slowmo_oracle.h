@@ -46,9 +46,12 @@ uint64_t oracle_stream_word(uint64_t key, uint64_t j);
 uint64_t oracle_stream_key(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, uint32_t w);
 /* Uniform in [0,1) with 24 bits from the top of a word; exact in binary32. */
 float oracle_word_to_unit(uint64_t r);
-/* One N(0,1) draw from one word: Box-Muller, cosine branch, binary32 arithmetic. */
-float oracle_word_to_normal(uint64_t r);
-/* Bulk export for tests: words and/or normals of one stream for j0 <= j < j0 + n. */
+/* Two independent N(0,1) draws from one word: Box-Muller (cosine, sine), binary32 arithmetic. */
+void oracle_word_to_normal_pair(uint64_t r, float z[2]);
+/* Normal of coordinate j in a stream: output (j & 1) of the pair made from word j >> 1. */
+float oracle_stream_normal(uint64_t key, uint64_t j);
+/* Bulk export for tests, for j0 <= j < j0 + n: words[i] = word j0+i of the stream,
+ * normals[i] = normal of coordinate j0+i (which is made from word (j0+i) >> 1). */
 void oracle_stream_export(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, uint32_t w,
                           uint64_t j0, uint64_t n, uint64_t *words, float *normals);
 

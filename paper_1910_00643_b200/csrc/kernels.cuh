@@ -36,14 +36,13 @@ fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t tag,
   const uint64_t key = stream_key(tag, seed, 0, 0, row);
   float *p = dst + (uint64_t)row * pitch;
   for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
-    uint64_t s = key + kGoldenGamma * (4 * vi + 1);
-    float4 o;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      comp(o, e) = __fmul_rn(scale, word_to_normal(mix64(s)));
-      s += kGoldenGamma;
-    }
-    st_stream(p + 4 * vi, o);
+    // columns 4vi..4vi+3 are the pairs 2vi and 2vi+1 of the row's stream
+    const uint64_t s = key + kGoldenGamma * (2 * vi + 1);
+    float4 z;
+    word_to_normal_pair(mix64(s), z.x, z.y);
+    word_to_normal_pair(mix64(s + kGoldenGamma), z.z, z.w);
+    st_stream(p + 4 * vi, make_float4(__fmul_rn(scale, z.x), __fmul_rn(scale, z.y), __fmul_rn(scale, z.z),
+                                      __fmul_rn(scale, z.w)));
   }
 }
 
@@ -73,13 +72,14 @@ fill_value_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, float value) {
     st_stream(p + 4 * vi, o);
 }
 
-// Export of one stream for the bit-exact test: words and/or normals for j0 <= j < j0 + n.
+// Export of one stream for the bit-exact test, j0 <= j < j0 + n: word j of the stream and/or
+// the normal of coordinate j.
 __global__ void __launch_bounds__(kThreads)
 export_stream_kernel(uint64_t key, uint64_t j0, uint64_t n, uint64_t *words, float *normals) {
   for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (uint64_t)gridDim.x * kThreads) {
     const uint64_t r = stream_word(key, j0 + i);
     if (words) words[i] = r;
-    if (normals) normals[i] = word_to_normal(r);
+    if (normals) normals[i] = stream_normal(key, j0 + i);
   }
 }
 
@@ -98,9 +98,26 @@ struct LocalArgs {
   float b1, b2, omb1, omb2, ibc1, ibc2, eps;  // Adam: betas, 1-betas, 1/(1-beta^l), epsilon
 };
 
+// One element of the base-optimizer step (Table C.1 direction, then Algorithm 1's update).
+template <int BASE>
+__device__ __forceinline__ void base_step(const LocalArgs &A, float g, float &x, float &h, float &v) {
+  if (A.wd != 0.0f) g = __fmaf_rn(A.wd, x, g);
+  float d;
+  if (BASE == 0) {
+    h = __fmaf_rn(A.mu, h, g);
+    d = __fmaf_rn(A.mu, h, g);
+  } else {
+    h = __fmaf_rn(A.b1, h, __fmul_rn(A.omb1, g));
+    v = __fmaf_rn(A.b2, v, __fmul_rn(A.omb2, __fmul_rn(g, g)));
+    d = __fdiv_rn(__fmul_rn(h, A.ibc1), __fadd_rn(__fsqrt_rn(__fmul_rn(v, A.ibc2)), A.eps));
+  }
+  x = __fmaf_rn(A.neg_gamma, d, x);
+}
+
 // One block = one tile of kThreads*U column groups of one row. Consecutive blocks are the m
 // rows of the same tile, so the shared curvature tile is read from DRAM once and from L2
-// m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic.
+// m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic;
+// the noise key of the row is derived by one lane per warp while those loads are in flight.
 template <int BASE, int GRAD, int U>
 __global__ void __launch_bounds__(kThreads)
 local_step_kernel(const LocalArgs A) {
@@ -108,12 +125,6 @@ local_step_kernel(const LocalArgs A) {
   const uint32_t tile = blockIdx.x / A.m;
   const uint32_t v0 = tile * (uint32_t)(kThreads * U) + threadIdx.x;
   const uint64_t roff = (uint64_t)row * A.pitch;
-
-  __shared__ uint64_t key_sh;
-  if (GRAD == 0) {
-    if (threadIdx.x == 0) key_sh = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
-    __syncthreads();
-  }
 
   float4 x[U], h[U], v[U], s[U], a[U];
   bool ok[U];
@@ -131,40 +142,31 @@ local_step_kernel(const LocalArgs A) {
     }
   }
 
+  uint64_t key = 0;
+  if (GRAD == 0) {
+    if ((threadIdx.x & 31u) == 0) key = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
+    key = __shfl_sync(0xFFFFFFFFu, key, 0);
+  }
+
 #pragma unroll
   for (int u = 0; u < U; ++u) {
     if (!ok[u]) continue;
     const uint32_t vi = v0 + u * kThreads;
-    uint64_t st = 0;
-    if (GRAD == 0) st = key_sh + kGoldenGamma * (4ull * vi + 1);
+    float4 g;
+    if (GRAD == 0) {
+      // columns 4vi..4vi+3 take the Box-Muller pairs of words 2vi and 2vi+1 of the row's stream
+      const uint64_t st = key + kGoldenGamma * (2ull * vi + 1);
+      float4 z;
+      word_to_normal_pair(mix64(st), z.x, z.y);
+      word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float xe = comp(x[u], e);
-      float g;
-      if (GRAD == 0) {
-        const float z = word_to_normal(mix64(st));
-        st += kGoldenGamma;
-        g = __fmaf_rn(comp(a[u], e), __fsub_rn(xe, comp(s[u], e)), __fmul_rn(A.sigma, z));
-      } else {
-        g = comp(s[u], e);
-      }
-      if (A.wd != 0.0f) g = __fmaf_rn(A.wd, xe, g);
-      float d;
-      if (BASE == 0) {
-        const float hn = __fmaf_rn(A.mu, comp(h[u], e), g);
-        d = __fmaf_rn(A.mu, hn, g);
-        comp(h[u], e) = hn;
-      } else {
-        const float hn = __fmaf_rn(A.b1, comp(h[u], e), __fmul_rn(A.omb1, g));
-        const float vn = __fmaf_rn(A.b2, comp(v[u], e), __fmul_rn(A.omb2, __fmul_rn(g, g)));
-        const float hh = __fmul_rn(hn, A.ibc1);
-        const float vh = __fmul_rn(vn, A.ibc2);
-        d = __fdiv_rn(hh, __fadd_rn(__fsqrt_rn(vh), A.eps));
-        comp(h[u], e) = hn;
-        comp(v[u], e) = vn;
-      }
-      comp(x[u], e) = __fmaf_rn(A.neg_gamma, d, xe);
+      for (int e = 0; e < 4; ++e)
+        comp(g, e) = __fmaf_rn(comp(a[u], e), __fsub_rn(comp(x[u], e), comp(s[u], e)), __fmul_rn(A.sigma, comp(z, e)));
+    } else {
+      g = s[u];
     }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) base_step<BASE>(A, comp(g, e), comp(x[u], e), comp(h[u], e), comp(v[u], e));
     const uint64_t off = roff + 4ull * vi;
     st_stream(A.x + off, x[u]);
     st_stream(A.h + off, h[u]);

@@ -76,19 +76,28 @@ def test_export_matches_single_word_calls_beyond_2_pow_32():
     L = oracle.lib()
     K = L.oracle_stream_key(3, 9, 4, 2, 1)
     assert [int(w) for w in words] == [L.oracle_stream_word(K, j0 + i) for i in range(8)]
-    assert all(z[i] == np.float32(L.oracle_word_to_normal(int(words[i]))) for i in range(8))
+    # coordinate j takes output j & 1 of the pair made from word j >> 1
+    for i in range(8):
+        j = j0 + i
+        pair = oracle.normal_pair(L.oracle_stream_word(K, j >> 1))
+        assert z[i] == np.float32(pair[j & 1])
+        assert z[i] == np.float32(L.oracle_stream_normal(K, j))
 
 
 def _libm_box_muller(words):
+    """Both Box-Muller outputs of each word in double precision: shape [n, 2]."""
     k1 = (words >> np.uint64(40)).astype(np.float64)
     k2 = ((words >> np.uint64(16)) & np.uint64(0xFFFFFF)).astype(np.float64)
-    u1 = (k1 + 1.0) / 2.0**24
-    return np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * k2 / 2.0**24)
+    radius = np.sqrt(-2.0 * np.log((k1 + 1.0) / 2.0**24))
+    angle = 2.0 * np.pi * k2 / 2.0**24
+    return np.stack([radius * np.cos(angle), radius * np.sin(angle)], axis=1)
 
 
 def test_normal_map_against_double_precision_box_muller():
-    words, z = oracle.stream(3, 0, 0, 0, 0, 0, 1 << 20)
-    ref = _libm_box_muller(words)
+    n = 1 << 20
+    words, z = oracle.stream(3, 0, 0, 0, 0, 0, n)
+    # coordinates 0..n-1 use words 0..n/2-1, cosine output first
+    ref = _libm_box_muller(words[: n // 2]).reshape(-1)
     err = np.abs(z.astype(np.float64) - ref)
     # binary32 evaluation: a few ulp of a value below 6, plus series truncation < 1e-8
     assert err.max() < 2e-6, err.max()
@@ -96,26 +105,41 @@ def test_normal_map_against_double_precision_box_muller():
 
 
 def test_normal_map_special_words():
-    L = oracle.lib()
-
     def word(k1, k2):
         return (k1 << 40) | (k2 << 16)
 
+    pair = oracle.normal_pair
     top = (1 << 24) - 1
     r_max = math.sqrt(2 * 24 * math.log(2))
-    assert L.oracle_word_to_normal(word(top, 12345)) == 0.0            # u1 = 1: radius 0
-    assert abs(L.oracle_word_to_normal(word(0, 0)) - r_max) < 1e-6       # u1 = 2^-24, angle 0
-    assert abs(L.oracle_word_to_normal(word(0, 1 << 23)) + r_max) < 1e-6  # angle pi
-    assert abs(L.oracle_word_to_normal(word(0, 1 << 22))) < 1e-6          # angle pi/2
-    assert abs(L.oracle_word_to_normal(word(0, 3 << 22))) < 1e-6          # angle 3pi/2
-    # angle pi/4 and its reflections in the other quadrants
-    c = r_max * math.sqrt(0.5)
-    for q, sign in ((0, 1), (1, -1), (2, -1), (3, 1)):
-        k2 = (q << 22) + (1 << 21) if q in (0, 2) else (q << 22) + (1 << 21)
-        got = L.oracle_word_to_normal(word(0, k2))
-        assert abs(got - sign * c) < 2e-6, (q, got)
+    assert pair(word(top, 12345)) == (0.0, 0.0)                           # u1 = 1: radius 0
+    for k2, c, s in ((0, 1, 0), (1 << 22, 0, 1), (1 << 23, -1, 0), (3 << 22, 0, -1)):
+        got = pair(word(0, k2))                                           # u1 = 2^-24, axis angles
+        assert abs(got[0] - c * r_max) < 1e-6 and abs(got[1] - s * r_max) < 1e-6, (k2, got)
+    # odd multiples of pi/4: both outputs have magnitude r_max / sqrt(2)
+    d = r_max * math.sqrt(0.5)
+    for q, (c, s) in enumerate(((1, 1), (-1, 1), (-1, -1), (1, -1))):
+        got = pair(word(0, (q << 22) + (1 << 21)))
+        assert abs(got[0] - c * d) < 2e-6 and abs(got[1] - s * d) < 2e-6, (q, got)
+    # just past pi/4 (reflected evaluation) in every quadrant
+    for q in range(4):
+        k2 = (q << 22) + (1 << 21) + 12345
+        ang = 2 * math.pi * k2 / 2**24
+        got = pair(word(0, k2))
+        assert abs(got[0] - r_max * math.cos(ang)) < 2e-6 and abs(got[1] - r_max * math.sin(ang)) < 2e-6
     # low 16 bits of the word are unused
-    assert L.oracle_word_to_normal(word(77, 99) | 0xFFFF) == L.oracle_word_to_normal(word(77, 99))
+    assert pair(word(77, 99) | 0xFFFF) == pair(word(77, 99))
+
+
+def test_pair_outputs_are_uncorrelated_and_jointly_normal():
+    n = 1 << 20
+    _, z = oracle.stream(3, 5, 1, 2, 0, 0, n)
+    zc, zs = z[0::2].astype(np.float64), z[1::2].astype(np.float64)
+    bound = 5.0 / math.sqrt(n // 2)
+    assert abs(np.corrcoef(zc, zs)[0, 1]) < bound
+    assert abs(np.corrcoef(zc**2, zs**2)[0, 1]) < bound   # independent, not merely uncorrelated
+    # z_c^2 + z_s^2 = -2 ln u1 is exponential with mean 2
+    r2 = zc**2 + zs**2
+    assert stats.kstest(r2[: 1 << 17], "expon", args=(0, 2.0)).pvalue > 1e-3
 
 
 def test_normal_and_uniform_distribution():
