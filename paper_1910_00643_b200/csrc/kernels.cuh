@@ -15,11 +15,29 @@ namespace slowmo {
 
 constexpr int kThreads = 256;
 
+// Tunables (overridable at compile time for parameter sweeps).
+#ifndef SLOWMO_LOCAL_UNROLL
+#define SLOWMO_LOCAL_UNROLL 2   // 128-bit column groups per thread in the local-step kernel
+#endif
+#ifndef SLOWMO_LOCAL_MIN_BLOCKS
+#define SLOWMO_LOCAL_MIN_BLOCKS 1  // __launch_bounds__ minimum resident blocks per SM
+#endif
+#ifndef SLOWMO_STREAM_HINT
+#define SLOWMO_STREAM_HINT 0    // 1: evict-first (.cs) loads and stores, 0: default policy
+#endif
+constexpr int kLocalUnroll = SLOWMO_LOCAL_UNROLL;
+
 // ---- streaming 128-bit accesses --------------------------------------------------------
-// Tensors are far larger than L2 and every line is used exactly once per launch, so loads
-// and stores carry the evict-first policy.
+// Tensors are far larger than L2 and every line is used exactly once per launch. The
+// evict-first policy (.cs) measured equal or slightly slower than the default on B200, so
+// the default policy is used; the hint stays selectable for sweeps.
+#if SLOWMO_STREAM_HINT
 __device__ __forceinline__ float4 ld_stream(const float *p) { return __ldcs(reinterpret_cast<const float4 *>(p)); }
 __device__ __forceinline__ void st_stream(float *p, float4 v) { __stcs(reinterpret_cast<float4 *>(p), v); }
+#else
+__device__ __forceinline__ float4 ld_stream(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st_stream(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+#endif
 // `a` is shared by the m rows of a column tile: keep it cacheable so the blocks of the other
 // rows, which run next to this one, find it in L2.
 __device__ __forceinline__ float4 ld_shared_row(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
@@ -119,7 +137,7 @@ __device__ __forceinline__ void base_step(const LocalArgs &A, float g, float &x,
 // m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic;
 // the noise key of the row is derived by one lane per warp while those loads are in flight.
 template <int BASE, int GRAD, int U>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, SLOWMO_LOCAL_MIN_BLOCKS)
 local_step_kernel(const LocalArgs A) {
   const uint32_t row = blockIdx.x % A.m;
   const uint32_t tile = blockIdx.x / A.m;

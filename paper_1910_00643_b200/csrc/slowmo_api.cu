@@ -35,8 +35,6 @@ struct slowmo_ctx {
 
 namespace {
 
-constexpr int kLocalUnroll = 2;
-
 bool finite_pos(float v) { return std::isfinite(v) && v > 0.0f; }
 bool unit_interval(float v) { return std::isfinite(v) && v >= 0.0f && v < 1.0f; }
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
