@@ -202,6 +202,50 @@ int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant);
  * bounded waits ran out (the record is then cleared), SLOWMO_ECUDA on a CUDA failure. */
 int slowmo_sync_status(slowmo_ctx *ctx);
 
+/*
+ * Outer step without a context and without any allocation. (The paper has no counterpart:
+ * this entry point exists for callers that must not allocate device memory.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a framework whose
+ * caching allocator owns all device memory and forbids raw allocations, in a process whose
+ * memory budget was fixed up front, or in a latency-critical loop where an allocation's
+ * implicit device synchronisation is unacceptable. slowmo_create cannot serve them,
+ * because it allocates the small status block that the staged (bulk-copy) outer-step
+ * kernel writes its bounded-wait record into. Here that scratch lives in a fixed 256-byte
+ * array inside the library image instead (every GPU that loads the library holds those 256
+ * bytes until the process exits), and all parameters that a context would remember are
+ * passed in.
+ *
+ * Computes exactly what slowmo_outer_step computes (same kernel, same arithmetic, same
+ * order): average of the m rows of x, Eq. (2), Eq. (3), broadcast, buffer policy, on the
+ * caller's device tensors x, h [m, pitch], v [m, pitch] (Adam only, else NULL), anchor,
+ * u [pitch], with the layout rules at the top of this file. base and buffer_policy are
+ * SLOWMO_BASE_* / SLOWMO_BUF_* (base only tells whether v exists).
+ *
+ * Limits: the scratch does not grow with the problem, so the only size limits are the
+ * kernel's index range: 1 <= P <= SLOWMO_STATIC_MAX_P and 1 <= m <= SLOWMO_STATIC_MAX_M;
+ * anything larger is refused with SLOWMO_EINVAL before any GPU work. Other errors as for
+ * slowmo_create / slowmo_outer_step (EINVAL, EALIGN, ECUDA).
+ *
+ * Set-up: the first call on each device (with that device current) looks up the scratch
+ * array's device address and raises the kernel's shared-memory limit. That first call
+ * should come before any stream capture. No call allocates or frees memory.
+ *
+ * Sharing: every call on a device uses the same scratch and clears it on the stream before
+ * its kernel. Calls that overlap on the GPU (different streams, or several host threads)
+ * race on it: their results stay correct, but a timeout record may be lost or attributed to
+ * the wrong call. Serialise calls if the record matters.
+ *
+ * wait != 0: the call waits for the stream and returns SLOWMO_ETIMEOUT if the kernel
+ * recorded that a bounded wait ran out (results are then invalid). wait == 0: the call
+ * returns once the work is enqueued.
+ */
+#define SLOWMO_STATIC_MAX_P ((1ull << 32) - 4096)
+#define SLOWMO_STATIC_MAX_M 65536u
+int slowmo_outer_step_static(float *x, float *h, float *v, float *anchor, float *u, uint64_t pitch,
+                             uint64_t P, uint32_t m, int32_t base, int32_t buffer_policy, float alpha,
+                             float beta, float gamma_t, void *cuda_stream, int wait);
+
 const char *slowmo_strerror(int status);
 int slowmo_last_cuda_error(slowmo_ctx *ctx);
 

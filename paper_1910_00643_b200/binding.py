@@ -23,7 +23,8 @@ VARIANT = {"default": 0, "direct": 1, "staged": 2}
 EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_outer_step",
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
-           "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error"]
+           "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
+           "slowmo_outer_step_static"]
 
 
 class SlowMoError(RuntimeError):
@@ -78,6 +79,8 @@ def lib():
             "slowmo_set_variant": [vp, C.c_int, C.c_int],
             "slowmo_sync_status": [vp],
             "slowmo_last_cuda_error": [vp],
+            "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
+                                         C.c_float, vp, C.c_int],
         }
         for name, args in sig.items():
             f = getattr(L, name)
@@ -113,6 +116,19 @@ def make_config(*, P, m, tau, alpha=1.0, beta=0.0, gamma=0.1, base="nesterov", m
         cfg.n_tensors = len(tensor_sizes)
         cfg.tensor_sizes = C.cast(arr, C.POINTER(C.c_uint64))
     return cfg
+
+
+def outer_step_static(x, h, v, anchor, u, *, pitch, P, m, base, buffer_policy, alpha, beta, gamma,
+                      stream=None, wait=True):
+    """slowmo_outer_step_static: the outer step on caller-owned torch CUDA tensors, for callers
+    that may not allocate device memory (no context, no cudaMalloc). Raises on any error."""
+    ptr = lambda t: None if t is None else t.data_ptr()
+    rc = lib().slowmo_outer_step_static(ptr(x), ptr(h), ptr(v), ptr(anchor), ptr(u), pitch, P, m,
+                                        BASE[base] if isinstance(base, str) else base,
+                                        POLICY[buffer_policy] if isinstance(buffer_policy, str) else buffer_policy,
+                                        alpha, beta, gamma, None if stream is None else stream.cuda_stream,
+                                        1 if wait else 0)
+    _check(rc, "slowmo_outer_step_static")
 
 
 def round_up(n, q):

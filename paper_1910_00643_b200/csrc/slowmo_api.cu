@@ -425,3 +425,100 @@ const char *slowmo_strerror(int status) {
 int slowmo_last_cuda_error(slowmo_ctx *ctx) { return ctx ? ctx->cuda_error : 0; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------
+// Allocation-free outer step (see slowmo_outer_step_static in include/slowmo.h).
+//
+// The staged outer-step kernel needs a few words of global scratch for its bounded-wait
+// record. A context gets them from cudaMalloc; callers that may not allocate get them from
+// this array, which is part of the library image on every device that loads it.
+//
+// In host code `g_static_scratch` is only a handle for the runtime, not a device address:
+// the address is looked up once per device with cudaGetSymbolAddress and that pointer is
+// what the kernel receives.
+// ---------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+
+constexpr int kStaticScratchInts = 64;  // 256 bytes; the kernel uses the first 4
+static __device__ __align__(256) int g_static_scratch[kStaticScratchInts];
+
+constexpr int kMaxDevices = 64;
+struct StaticDeviceState {
+  int *scratch = nullptr;  // device address of g_static_scratch on this device
+  int num_sms = 0;
+};
+StaticDeviceState g_static_state[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: resolve the scratch address, raise the staged
+// kernel's dynamic shared-memory limit, read the SM count. Allocates nothing.
+cudaError_t static_setup(int dev, StaticDeviceState **out) {
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticDeviceState &st = g_static_state[dev];
+  if (!st.scratch) {
+    int *ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!ptr) return cudaErrorInvalidSymbol;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = outer_staged_configure();
+    if (e != cudaSuccess) return e;
+    st.num_sms = sms;
+    st.scratch = ptr;
+  }
+  *out = &st;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int slowmo_outer_step_static(float *x, float *h, float *v, float *anchor, float *u, uint64_t pitch,
+                                        uint64_t P, uint32_t m, int32_t base, int32_t buffer_policy, float alpha,
+                                        float beta, float gamma_t, void *cuda_stream, int wait) {
+  const bool adam = base == SLOWMO_BASE_ADAM;
+  if (base != SLOWMO_BASE_NESTEROV && !adam) return SLOWMO_EINVAL;
+  if (buffer_policy < SLOWMO_BUF_RESET || buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
+  if (P == 0 || P > SLOWMO_STATIC_MAX_P || m == 0 || m > SLOWMO_STATIC_MAX_M) return SLOWMO_EINVAL;
+  if (!finite_pos(alpha) || !unit_interval(beta) || !finite_pos(gamma_t)) return SLOWMO_EINVAL;
+  if (!x || !h || !anchor || !u || (adam && !v)) return SLOWMO_EINVAL;
+  if (pitch % 4 != 0) return SLOWMO_EALIGN;
+  if (pitch < P) return SLOWMO_EINVAL;
+  const void *ptrs[] = {x, h, v, anchor, u};
+  for (const void *p : ptrs)
+    if (p && !aligned16(p)) return SLOWMO_EALIGN;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SLOWMO_ECUDA;
+  StaticDeviceState *st = nullptr;
+  if (static_setup(dev, &st) != cudaSuccess) return SLOWMO_ECUDA;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+  OuterArgs A;
+  A.x = x;
+  A.h = h;
+  A.v = v;
+  A.anchor = anchor;
+  A.u = u;
+  A.pitch = pitch;
+  A.nvec = (uint32_t)((P + 3) / 4);
+  A.m = m;
+  A.beta = beta;
+  A.inv_gamma = (float)(1.0 / (double)gamma_t);
+  A.neg_alpha_gamma = -(float)((double)alpha * (double)gamma_t);
+  A.m_float = (float)m;
+
+  // the scratch keeps the previous call's record: clear the words the kernel reads
+  if (cudaMemsetAsync(st->scratch, 0, 4 * sizeof(int), stream) != cudaSuccess) return SLOWMO_ECUDA;
+  launch_outer_staged(A, adam ? 2 : 1, buffer_policy, st->num_sms, st->scratch, stream);
+  if (cudaGetLastError() != cudaSuccess) return SLOWMO_ECUDA;
+  if (!wait) return SLOWMO_OK;
+
+  int host[4] = {0, 0, 0, 0};
+  if (cudaMemcpyAsync(host, st->scratch, sizeof(host), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return SLOWMO_ECUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return SLOWMO_ECUDA;
+  return host[0] != 0 ? SLOWMO_ETIMEOUT : SLOWMO_OK;
+}
