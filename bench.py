@@ -26,9 +26,12 @@ METRIC = "replica-param updates/sec (local + outer step)"
 UNIT = "updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram bytes per launch measured with ncu for the dominant kernel (see profiles/); None until
-# a capture of the current kernel exists
-NCU_TRAFFIC_BYTES = {"local_step": None, "outer_step": None}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch divided by the
+# algorithmic bytes, from ncu captures of small cases of the current kernels (profiles/);
+# traffic grows in proportion to m*P, so the ratio carries to the full launch. None = no capture
+# of the kernel as it stands.
+NCU_TRAFFIC_RATIO = {("local_step", "generated"): 0.962, ("local_step", "supplied"): 0.980,
+                     ("outer_step", "average"): 0.951, ("outer_step", "reset"): 0.973}
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -213,13 +216,16 @@ def time_steps_e2e(s, w, steps, warmup, host_in, host_out, which_in, grad=None):
     return max(wall_ms, dev_ms)
 
 
-def roofline(kind, bytes_per_launch, ms, peak, peak_kind):
+def roofline(kind, bytes_per_launch, ms, peak, peak_kind, case=None):
     achieved = bytes_per_launch / (ms * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_RATIO.get((kind, case))
     return {"bound": "hbm", "kernel": kind, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
             "frac": round(achieved / peak, 4), "peak_kind": peak_kind + " copy bandwidth",
             "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
             "bytes_per_launch": bytes_per_launch, "ms_per_launch": round(ms, 4),
-            "traffic": NCU_TRAFFIC_BYTES.get(kind)}
+            "traffic": None if ratio is None else int(ratio * bytes_per_launch),
+            "traffic_source": None if ratio is None else
+            f"ncu small-case capture scaled by m*P (traffic / algorithmic = {ratio})"}
 
 
 def cpu_baseline(w, budget_s=15.0):
@@ -252,8 +258,9 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
     for variant in ("direct", "staged"):
         s.set_variant("outer", variant)
         total, local, outer = time_steps(s, w, iters, 1, s.grad)
-        out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind)
-        out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind)
+        out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind, "supplied")
+        out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind,
+                                                "reset" if variant == "direct" else None)
         out["updates_per_s_tau%d_%s" % (tau, variant)] = w["m"] * w["P"] * tau * iters / (total * 1e-3)
     s.close()
     del s
@@ -334,8 +341,11 @@ def run_ours(args):
                    "l2": "state tensors (>= 5 GB) are far larger than the 126 MB L2; no flush needed"},
         "gpu_launches": args.steps * (w["tau"] + 1),
         "clocks": clocks,
-        "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind),
-        "roofline_outer_step": roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind),
+        "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
+                             w["grad_mode"] if w["base"] == "nesterov" else None),
+        "roofline_outer_step": roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
+                                        w["buffer_policy"] if args.outer_variant in (None, "direct")
+                                        and w["base"] == "nesterov" and w["buffer_policy"] != "maintain" else None),
         "e2e": e2e,
     }
     if rank == 0 and world == 1:
