@@ -103,6 +103,8 @@ export_stream_kernel(uint64_t key, uint64_t j0, uint64_t n, uint64_t *words, flo
 
 // ---- K1: fused multi-replica base-optimizer step ------------------------------------------
 
+constexpr uint32_t kInlineKeys = 64;  // noise keys of up to this many rows travel in the kernel arguments
+
 struct LocalArgs {
   float *x, *h, *v;       // [m, pitch]
   const float *src;       // generated mode: centres c [m, pitch]; supplied mode: gradient G [m, pitch]
@@ -114,6 +116,7 @@ struct LocalArgs {
   uint32_t k;             // inner step, for the noise key
   float neg_gamma, mu, wd, sigma;
   float b1, b2, omb1, omb2, ibc1, ibc2, eps;  // Adam: betas, 1-betas, 1/(1-beta^l), epsilon
+  uint64_t keys[kInlineKeys];  // generated mode, m <= kInlineKeys: stream key of (t, k, row), host-computed
 };
 
 // One element of the base-optimizer step (Table C.1 direction, then Algorithm 1's update).
@@ -134,8 +137,10 @@ __device__ __forceinline__ void base_step(const LocalArgs &A, float g, float &x,
 
 // One block = one tile of kThreads*U column groups of one row. Consecutive blocks are the m
 // rows of the same tile, so the shared curvature tile is read from DRAM once and from L2
-// m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic;
-// the noise key of the row is derived by one lane per warp while those loads are in flight.
+// m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic.
+// The noise key of the row comes with the kernel arguments (computed on the host, the same
+// integer arithmetic) so that no issue slot is spent on it; beyond kInlineKeys rows it is
+// derived in the kernel.
 template <int BASE, int GRAD, int U>
 __global__ void __launch_bounds__(kThreads, SLOWMO_LOCAL_MIN_BLOCKS)
 local_step_kernel(const LocalArgs A) {
@@ -162,8 +167,12 @@ local_step_kernel(const LocalArgs A) {
 
   uint64_t key = 0;
   if (GRAD == 0) {
-    if ((threadIdx.x & 31u) == 0) key = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
-    key = __shfl_sync(0xFFFFFFFFu, key, 0);
+    if (A.m <= kInlineKeys) {
+      key = A.keys[row];
+    } else {  // many workers: one lane per warp derives the key while the loads are in flight
+      if ((threadIdx.x & 31u) == 0) key = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
+      key = __shfl_sync(0xFFFFFFFFu, key, 0);
+    }
   }
 
 #pragma unroll

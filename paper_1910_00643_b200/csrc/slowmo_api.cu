@@ -272,6 +272,8 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     A.ibc2 = (float)(1.0 / (1.0 - ctx->pow_b2));
     A.t = ctx->t;
     A.k = ctx->k;
+    if (generated && c.m <= kInlineKeys)
+      for (uint32_t i = 0; i < c.m; ++i) A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, i);
     if (c.base == SLOWMO_BASE_NESTEROV) {
       if (generated) launch_local<0, 0>(ctx, A); else launch_local<0, 1>(ctx, A);
     } else {

@@ -164,6 +164,16 @@ def test_many_workers():
         s.close()
 
 
+def test_more_workers_than_inline_noise_keys():
+    # beyond 64 workers the local-step kernel derives its noise keys itself
+    w = workloads.workload("tiny", P=1030, m=70, tau=2, T=2, buffer_policy="maintain")
+    s = _slowmo(w, guard=64)
+    s.run(2)
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+
+
 def test_every_worker_holds_the_anchor_after_the_outer_step():
     import torch
     w = workloads.workload("tiny", P=10_001, m=6)
