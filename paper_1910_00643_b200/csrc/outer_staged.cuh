@@ -2,11 +2,13 @@
 // broadcast, buffer policy) with the replica rows moved by the bulk-copy engine (TMA).
 //
 // A persistent CTA owns column tiles of kTileCols columns. For each tile a producer thread
-// streams the m row segments into a ring of shared-memory stages with
+// streams the m row segments (and, with the first of them, the anchor and u tiles) into a
+// ring of shared-memory stages with
 // cp.async.bulk (global -> shared, completion on an mbarrier); eight consumer warps add the
 // rows in worker order, apply Eq. (2)/(3), put the new anchor tile in shared memory once and
-// one thread sends it to all m replica rows (and the anchor) with m+1 bulk stores
-// (shared -> global). The buffer policy reuses the same machinery: "reset" bulk-stores a
+// a store thread sends it to all m replica rows (and the anchor) with m+1 bulk stores
+// (shared -> global); consumers and store thread hand tiles over through mbarriers, so no
+// CTA-wide barrier sits in the loop. The buffer policy reuses the same machinery: "reset" bulk-stores a
 // zero tile, "average" streams the h (and v) rows through the ring like x.
 //
 // No cluster multicast is used anywhere; every copy is CTA-local and starts on a 16-byte
@@ -25,20 +27,38 @@
 namespace slowmo {
 
 constexpr int kTileCols = 1024;                    // columns per tile: 4 per consumer thread
-constexpr int kStageRows = 4;                      // row segments per pipeline stage
-constexpr int kStages = 6;                         // ring depth
+#ifndef SLOWMO_STAGED_ROWS
+#define SLOWMO_STAGED_ROWS 4
+#endif
+#ifndef SLOWMO_STAGED_STAGES
+#define SLOWMO_STAGED_STAGES 4
+#endif
+#ifndef SLOWMO_STAGED_CTAS
+#define SLOWMO_STAGED_CTAS 2
+#endif
+constexpr int kStageRows = SLOWMO_STAGED_ROWS;     // row segments per pipeline stage
+constexpr int kStages = SLOWMO_STAGED_STAGES;      // ring depth
+#ifndef SLOWMO_STAGED_BULK_STORES
+#define SLOWMO_STAGED_BULK_STORES 1  // 1: rows written by bulk copies from shared memory; 0: by vector stores
+#endif
+constexpr int kOutBufs = 3;                        // output tiles in flight per CTA
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kStagedThreads = kConsumerThreads + 32;  // + one producer warp
+constexpr int kStagedThreads = kConsumerThreads + 64;  // + one load-producer warp + one store warp
 constexpr uint32_t kWaitTries = 1u << 20;          // bound of every mbarrier wait
-constexpr int kStagedCtasPerSm = 2;
+constexpr int kStagedCtasPerSm = SLOWMO_STAGED_CTAS;
+
+constexpr int kAnchorSlot = kStageRows;            // extra slots of a stage: anchor and u tiles,
+constexpr int kUSlot = kStageRows + 1;             // filled with the first row chunk of each tile
 
 struct StagedSmem {
-  float stage[kStages][kStageRows][kTileCols];
-  float out[2][kTileCols];
+  float stage[kStages][kStageRows + 2][kTileCols];
+  float out[kOutBufs][kTileCols];
   float zeros[kTileCols];
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
+  unsigned long long out_full[kOutBufs];   // consumers -> store thread: tile written
+  unsigned long long out_empty[kOutBufs];  // store thread -> consumers: bulk stores have read the tile
   volatile int abort;
 };
 
@@ -92,7 +112,6 @@ __device__ __forceinline__ void bulk_wait_read() {
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory"); }
 
 // NBUF: base-optimizer buffers (1: h; 2: h, v). POLICY: 0 reset, 1 maintain, 2 average.
 template <int NBUF, int POLICY>
@@ -113,6 +132,10 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
       mbar_init(&S.full[s], 1);
       mbar_init(&S.empty[s], kConsumerWarps);
     }
+    for (int b = 0; b < kOutBufs; ++b) {
+      mbar_init(&S.out_full[b], kConsumerWarps);
+      mbar_init(&S.out_empty[b], 1);
+    }
     S.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -121,37 +144,39 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
   __syncthreads();
 
   if (warp == kConsumerWarps) {
-    // ---------------- producer: one thread feeds the ring ----------------
-    if ((tid & 31) == 0) {
-      uint32_t job = 0, issued = 0;  // issued: jobs whose copies were started
-      for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const uint32_t col0 = tile * kTileCols;
-        const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
-        for (int pass = 0; pass < kPasses; ++pass) {
-          const float *src = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
-          for (uint32_t c = 0; c < nchunks; ++c, ++job) {
-            const uint32_t st = job % kStages, round = job / kStages;
-            mbar_wait(&S.empty[st], (round & 1u) ^ 1u, &S.abort, status, 1);
-            if (S.abort) continue;
-            issued = job + 1;
-            const uint32_t r0 = c * kStageRows;
-            const uint32_t rows = min((uint32_t)kStageRows, A.m - r0);
-            mbar_expect_tx(&S.full[st], rows * ncols * 4u);
-            for (uint32_t r = 0; r < rows; ++r)
-              bulk_load(&S.stage[st][r][0], src + (uint64_t)(r0 + r) * A.pitch + col0, ncols * 4u, &S.full[st]);
-          }
+    // ---------------- producer warp: feeds the ring, one lane per row segment ----------------
+    const uint32_t lane = tid & 31u;
+    uint32_t job = 0, issued = 0;  // issued: jobs whose copies were started
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const uint32_t col0 = tile * kTileCols;
+      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      for (int pass = 0; pass < kPasses; ++pass) {
+        const float *src = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
+        for (uint32_t c = 0; c < nchunks; ++c, ++job) {
+          const uint32_t st = job % kStages, round = job / kStages;
+          if (lane == 0) mbar_wait(&S.empty[st], (round & 1u) ^ 1u, &S.abort, status, 1);
+          __syncwarp();
+          if (S.abort) continue;
+          issued = job + 1;
+          const uint32_t r0 = c * kStageRows;
+          const uint32_t rows = min((uint32_t)kStageRows, A.m - r0);
+          const bool first = pass == 0 && c == 0;  // this chunk also brings the anchor and u tiles
+          if (lane == 0) mbar_expect_tx(&S.full[st], (rows + (first ? 2u : 0u)) * ncols * 4u);
+          if (lane < rows)
+            bulk_load(&S.stage[st][lane][0], src + (uint64_t)(r0 + lane) * A.pitch + col0, ncols * 4u, &S.full[st]);
+          if (first && lane == kAnchorSlot) bulk_load(&S.stage[st][kAnchorSlot][0], A.anchor + col0, ncols * 4u, &S.full[st]);
+          if (first && lane == kUSlot) bulk_load(&S.stage[st][kUSlot][0], A.u + col0, ncols * 4u, &S.full[st]);
         }
       }
-      // copies still in flight must land before the shared memory is given back
-      if (S.abort) {
-        for (uint32_t j = issued > (uint32_t)kStages ? issued - kStages : 0; j < issued; ++j)
-          for (uint32_t i = 0; i < kWaitTries; ++i)
-            if (mbar_try_wait(&S.full[j % kStages], (j / kStages) & 1u)) break;
-      }
     }
-  } else {
+    // copies still in flight must land before the shared memory is given back
+    if (S.abort && lane == 0) {
+      for (uint32_t j = issued > (uint32_t)kStages ? issued - kStages : 0; j < issued; ++j)
+        for (uint32_t i = 0; i < kWaitTries; ++i)
+          if (mbar_try_wait(&S.full[j % kStages], (j / kStages) & 1u)) break;
+    }
+  } else if (warp < kConsumerWarps) {
     // ---------------- consumers ----------------
-    const bool issuer = tid == 0;
     uint32_t job = 0, outs = 0;
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
       const uint32_t col0 = tile * kTileCols;
@@ -160,10 +185,6 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
       const uint64_t col = (uint64_t)col0 + tid * 4u;
 
       float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), u0 = x0;
-      if (active) {
-        x0 = ld_stream(A.anchor + col);
-        u0 = ld_stream(A.u + col);
-      }
 
       for (int pass = 0; pass < kPasses; ++pass) {
         // ordered sum over the workers, chunk by chunk
@@ -173,6 +194,10 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
           mbar_wait(&S.full[st], round & 1u, &S.abort, status, 2);
           const uint32_t rows = min((uint32_t)kStageRows, A.m - c * kStageRows);
           if (active) {
+            if (pass == 0 && c == 0) {
+              x0 = *reinterpret_cast<const float4 *>(&S.stage[st][kAnchorSlot][tid * 4u]);
+              u0 = *reinterpret_cast<const float4 *>(&S.stage[st][kUSlot][tid * 4u]);
+            }
 #pragma unroll
             for (int r = 0; r < kStageRows; ++r) {
               if ((uint32_t)r < rows) {
@@ -206,30 +231,62 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
           if (active && !S.abort) st_stream(A.u + col, un);
         }
 
-        // the tile goes to shared memory once and from there to every row
-        const uint32_t ob = outs & 1u;
-        ++outs;
-        if (issuer) bulk_wait_read<1>();  // the bulk stores that last read out[ob] are done with it
-        consumer_sync();
-        if (active) *reinterpret_cast<float4 *>(&S.out[ob][tid * 4u]) = outv;
-        fence_async_proxy();
-        consumer_sync();
-        if (issuer && !S.abort) {
+#if !SLOWMO_STAGED_BULK_STORES
+        if (active && !S.abort) {
           float *dst = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
-          for (uint32_t i = 0; i < A.m; ++i) bulk_store(dst + (uint64_t)i * A.pitch + col0, &S.out[ob][0], ncols * 4u);
+          store_rows(dst + col, A.pitch, A.m, outv);
           if (pass == 0) {
-            bulk_store(A.anchor + col0, &S.out[ob][0], ncols * 4u);
-            if (POLICY == 0) {  // reset: zero tiles to every buffer row
-              for (uint32_t i = 0; i < A.m; ++i) bulk_store(A.h + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
-              if (NBUF == 2)
-                for (uint32_t i = 0; i < A.m; ++i) bulk_store(A.v + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
+            st_stream(A.anchor + col, outv);
+            if (POLICY == 0) {
+              const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+              store_rows(A.h + col, A.pitch, A.m, zero);
+              if (NBUF == 2) store_rows(A.v + col, A.pitch, A.m, zero);
             }
           }
-          bulk_commit();
         }
+        continue;
+#endif
+        // the tile goes to shared memory once; the store warp sends it to every row
+        const uint32_t ob = outs % kOutBufs, oround = outs / kOutBufs;
+        ++outs;
+        mbar_wait(&S.out_empty[ob], (oround & 1u) ^ 1u, &S.abort, status, 3);
+        if (active) *reinterpret_cast<float4 *>(&S.out[ob][tid * 4u]) = outv;
+        fence_async_proxy();
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(&S.out_full[ob]);
       }
     }
-    if (issuer) bulk_wait_all();
+  } else if (SLOWMO_STAGED_BULK_STORES && warp == kConsumerWarps + 1) {
+    // ---------------- store warp: output tiles -> all rows, lanes share the rows ----------------
+    const uint32_t lane = tid & 31u;
+    uint32_t outs = 0;
+    for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+      const uint32_t col0 = tile * kTileCols;
+      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      for (int pass = 0; pass < kPasses; ++pass, ++outs) {
+        const uint32_t ob = outs % kOutBufs, oround = outs / kOutBufs;
+        if (lane == 0) mbar_wait(&S.out_full[ob], oround & 1u, &S.abort, status, 4);
+        __syncwarp();
+        if (!S.abort) {
+          float *dst = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
+          for (uint32_t i = lane; i < A.m; i += 32) {
+            bulk_store(dst + (uint64_t)i * A.pitch + col0, &S.out[ob][0], ncols * 4u);
+            if (pass == 0 && POLICY == 0) {  // reset: zero tiles to every buffer row
+              bulk_store(A.h + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
+              if (NBUF == 2) bulk_store(A.v + (uint64_t)i * A.pitch + col0, &S.zeros[0], ncols * 4u);
+            }
+          }
+          if (pass == 0 && lane == 31) bulk_store(A.anchor + col0, &S.out[ob][0], ncols * 4u);
+        }
+        bulk_commit();
+        // every lane waits for its own groups: all but the newest kOutBufs-1 have been read out
+        // of shared memory, so the tile written kOutBufs-1 outputs ago can be overwritten
+        bulk_wait_read<kOutBufs - 1>();
+        __syncwarp();
+        if (lane == 0 && outs + 1 >= (uint32_t)kOutBufs) mbar_arrive(&S.out_empty[(outs + 1) % kOutBufs]);
+      }
+    }
+    bulk_wait_all();
   }
   __syncthreads();
 }
