@@ -61,6 +61,19 @@ def outer_step_bytes(w):
     return per_param * P
 
 
+def fused_outer_step_bytes(w):
+    """Algorithmic HBM bytes of the outer-step kernel that also takes the last inner step.
+    Per parameter: x, h [, v] and c-or-G of the m rows read, a, anchor, u read; u, anchor and
+    the m rows of x written; the m rows of h [, v] written once under every policy (stepped
+    values, zeros or means)."""
+    m, P = w["m"], w["P"]
+    nb = 2 if w["base"] == "adam" else 1
+    per_param = m * (4 + 4 * nb + 4) + 8 + 8 + m * 4 + m * 4 * nb
+    if w["grad_mode"] == "generated":
+        per_param += 4
+    return per_param * P
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -160,9 +173,12 @@ def aggregate_throughput(units_this_rank, ms_this_rank, device=None):
 
 # --------------------------------------------------------------------------------- timed loops
 
-def time_steps(s, w, steps, warmup, grad=None):
-    """Device-timed outer iterations. Returns total ms and the per-kernel mean launch ms."""
+def time_steps(s, w, steps, warmup, grad=None, fused=False):
+    """Device-timed outer iterations. Returns total ms and the per-kernel mean launch ms.
+    With the fused variant the last inner step runs inside the outer-step kernel, so an
+    iteration has tau-1 local-step launches."""
     import torch
+    local_launches = max(1, w["tau"] - 1) if fused else w["tau"]
     for _ in range(warmup):
         s.local_steps(w["tau"], grad)
         s.outer_step()
@@ -180,7 +196,7 @@ def time_steps(s, w, steps, warmup, grad=None):
     torch.cuda.synchronize()
     barrier()
     total = ev[0][0].elapsed_time(ev[-1][2])
-    local = sum(e[0].elapsed_time(e[1]) for e in ev) / (steps * w["tau"])
+    local = sum(e[0].elapsed_time(e[1]) for e in ev) / (steps * local_launches)
     outer = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
     s.sync_status()
     return total, local, outer
@@ -255,12 +271,16 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
     s = SlowMo(w)
     s.alloc_gradient()
     s.fill_gradient()
-    for variant in ("direct", "staged"):
+    for variant in ("direct", "staged", "fused"):
         s.set_variant("outer", variant)
-        total, local, outer = time_steps(s, w, iters, 1, s.grad)
-        out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind, "supplied")
-        out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind,
-                                                "reset" if variant == "direct" else None)
+        total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant == "fused")
+        if variant == "fused":
+            out["last_step_outer_fused"] = roofline("last_step_outer", fused_outer_step_bytes(w), outer, peak,
+                                                    peak_kind)
+        else:
+            out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind, "supplied")
+            out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind,
+                                                    "reset" if variant == "direct" else None)
         out["updates_per_s_tau%d_%s" % (tau, variant)] = w["m"] * w["P"] * tau * iters / (total * 1e-3)
     s.close()
     del s
@@ -297,8 +317,8 @@ def run_ours(args):
     w = workloads.workload(args.workload, **size_overrides(args))
     peak, peak_kind = measured_peak()
     s = SlowMo(w)
-    if args.outer_variant:
-        s.set_variant("outer", args.outer_variant)
+    s.set_variant("outer", args.outer_variant)
+    fused = args.outer_variant == "fused" and (w["grad_mode"] == "supplied" or w["m"] <= 64) and w["tau"] > 1
     grad = None
     if w["grad_mode"] == "supplied":
         grad = s.alloc_gradient()
@@ -306,7 +326,7 @@ def run_ours(args):
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, local_ms, outer_ms = time_steps(s, w, args.steps, args.warmup, grad)
+    total_ms, local_ms, outer_ms = time_steps(s, w, args.steps, args.warmup, grad, fused=fused)
     clocks = sampler.stop()
     units = w["m"] * w["P"] * w["tau"] * args.steps
     value, ms = aggregate_throughput(units, total_ms, dev)
@@ -336,16 +356,21 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{args.workload}: P={w['P']} m={w['m']} tau={w['tau']} "
                                f"base={w['base']} buffers={w['buffer_policy']} grad={w['grad_mode']}",
-                   "step": "one outer iteration = tau local-step launches + one outer-step launch",
+                   "step": ("one outer iteration = tau-1 local-step launches + one launch of the outer step "
+                            "with the last inner step fused in (SLOWMO_OUTER_FUSED)") if fused else
+                           "one outer iteration = tau local-step launches + one outer-step launch",
+                   "outer_variant": args.outer_variant,
                    "replicas": "independent replica of the workload per GPU, no collective on the data path",
                    "l2": "state tensors (>= 5 GB) are far larger than the 126 MB L2; no flush needed"},
-        "gpu_launches": args.steps * (w["tau"] + 1),
+        "gpu_launches": args.steps * (w["tau"] + (0 if fused else 1)),
         "clocks": clocks,
         "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
                              w["grad_mode"] if w["base"] == "nesterov" else None),
-        "roofline_outer_step": roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
-                                        w["buffer_policy"] if args.outer_variant in (None, "direct")
-                                        and w["base"] == "nesterov" and w["buffer_policy"] != "maintain" else None),
+        "roofline_outer_step": (
+            roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind) if fused else
+            roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
+                     w["buffer_policy"] if args.outer_variant == "direct" and w["base"] == "nesterov"
+                     and w["buffer_policy"] != "maintain" else None)),
         "e2e": e2e,
     }
     if rank == 0 and world == 1:
@@ -401,7 +426,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50")
-    ap.add_argument("--outer-variant", default=None, choices=[None, "direct", "staged"])
+    ap.add_argument("--outer-variant", default="fused", choices=["direct", "staged", "fused"])
     ap.add_argument("--P", type=int, default=None, help="override the workload's parameter count")
     ap.add_argument("--m", type=int, default=None, help="override the workload's worker count")
     ap.add_argument("--tau", type=int, default=None, help="override the workload's inner steps")

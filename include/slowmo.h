@@ -68,7 +68,10 @@ enum { SLOWMO_K_LOCAL = 0, SLOWMO_K_OUTER = 1 };
 enum {
   SLOWMO_VARIANT_DEFAULT = 0,
   SLOWMO_OUTER_DIRECT = 1, /* vector loads straight to registers                      */
-  SLOWMO_OUTER_STAGED = 2  /* bulk-copy (TMA) staging of row tiles through shared mem  */
+  SLOWMO_OUTER_STAGED = 2, /* bulk-copy (TMA) staging of row tiles through shared mem  */
+  SLOWMO_OUTER_FUSED = 3   /* the last inner step of each outer iteration runs inside the
+                              outer-step kernel (same results, fewer HBM bytes); see
+                              slowmo_local_steps for what this changes for the caller       */
 };
 
 /*
@@ -140,6 +143,14 @@ int slowmo_destroy(slowmo_ctx *ctx);
  *
  * `grad` is a device [m, pitch] tensor in supplied mode (read by each of the n steps) and
  * must be NULL in generated mode (EINVAL otherwise).
+ *
+ * With the SLOWMO_OUTER_FUSED variant selected, the step that completes the outer iteration
+ * (k = tau-1) is not launched here: it is taken inside slowmo_outer_step's kernel. Until
+ * then the caller's x, h, v tensors hold the state before that step, and in supplied mode
+ * `grad` must stay valid and unchanged until slowmo_outer_step has been enqueued. Every
+ * library call that reads or writes state (slowmo_get_params, slowmo_set_params,
+ * slowmo_sync_status, slowmo_set_variant, slowmo_destroy) first runs the deferred step, so
+ * results seen through the API are the same as without the variant.
  */
 int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad);
 

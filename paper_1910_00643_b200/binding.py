@@ -19,7 +19,7 @@ POLICY = {"reset": 0, "maintain": 1, "average": 2}
 GRAD = {"generated": 0, "supplied": 1}
 TENSOR = {"x": 0, "anchor": 1, "u": 2, "h": 3, "v": 4, "a": 5, "c": 6}
 KERNEL = {"local": 0, "outer": 1}
-VARIANT = {"default": 0, "direct": 1, "staged": 2}
+VARIANT = {"default": 0, "direct": 1, "staged": 2, "fused": 3}
 EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_outer_step",
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",

@@ -1,0 +1,132 @@
+// K2 with the last inner step folded in: the base-optimizer step k = tau-1 of every worker
+// (Table C.1 direction, Algorithm 1 update) is taken in registers and followed at once by
+// the exact average, Eq. (2), Eq. (3), the broadcast and the buffer policy.
+//
+// Same arithmetic, in the same order, as local_step_kernel followed by
+// outer_step_direct_kernel, so results are bit-identical; what disappears is one round trip
+// of x (and of h, v when they are reset or averaged) through HBM: per parameter
+//   separate: (20m + 4) + (8m + 16) + policy     fused: 20m + 16 + 4  (+8m for Adam's v)
+// with policy = 0 / 4m nb / 8m nb bytes for maintain / reset / average.
+#pragma once
+#include "kernels.cuh"
+
+namespace slowmo {
+
+__device__ __forceinline__ void add_in_order(float4 &s, const float4 &v, bool first) {
+  if (first) {
+    s = v;
+  } else {
+    s.x = __fadd_rn(s.x, v.x);
+    s.y = __fadd_rn(s.y, v.y);
+    s.z = __fadd_rn(s.z, v.z);
+    s.w = __fadd_rn(s.w, v.w);
+  }
+}
+
+__device__ __forceinline__ float4 div4(const float4 &s, float d) {
+  return make_float4(__fdiv_rn(s.x, d), __fdiv_rn(s.y, d), __fdiv_rn(s.z, d), __fdiv_rn(s.w, d));
+}
+
+// One thread = one 4-element column group, all m rows. ROWS rows are loaded together.
+// Requires m <= kInlineKeys in generated mode (the launcher falls back otherwise).
+template <int BASE, int GRAD, int POLICY, int ROWS>
+__global__ void __launch_bounds__(kThreads)
+last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
+  const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
+  if (vi >= O.nvec) return;
+  const uint64_t col = 4ull * vi;
+  const uint32_t m = O.m;
+
+  const float4 x0 = ld_stream(O.anchor + col);
+  const float4 u0 = ld_stream(O.u + col);
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (GRAD == 0) a = ld_shared_row(L.a + col);
+
+  float4 sx = a, sh = a, sv = a;  // ordered sums over the workers (overwritten at row 0)
+  for (uint32_t i0 = 0; i0 < m; i0 += ROWS) {
+    float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) {
+      if (i0 + q < m) {
+        const uint64_t off = (uint64_t)(i0 + q) * O.pitch + col;
+        x[q] = ld_stream(L.x + off);
+        h[q] = ld_stream(L.h + off);
+        if (BASE == 1) v[q] = ld_stream(L.v + off);
+        s[q] = ld_stream(L.src + off);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) {
+      const uint32_t i = i0 + q;
+      if (i >= m) break;
+      float4 g;
+      if (GRAD == 0) {
+        const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * vi + 1);
+        float4 z;
+        word_to_normal_pair(mix64(st), z.x, z.y);
+        word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(L.sigma, comp(z, e)));
+      } else {
+        g = s[q];
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
+      add_in_order(sx, x[q], i == 0);
+      if (POLICY == 1) {  // maintain: the stepped buffers go back to their rows
+        const uint64_t off = (uint64_t)i * O.pitch + col;
+        st_stream(L.h + off, h[q]);
+        if (BASE == 1) st_stream(L.v + off, v[q]);
+      } else if (POLICY == 2) {  // average
+        add_in_order(sh, h[q], i == 0);
+        if (BASE == 1) add_in_order(sv, v[q], i == 0);
+      }
+    }
+  }
+
+  const float4 xbar = div4(sx, O.m_float);
+  float4 un, xn;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    // Eq. (2): u <- beta u + (x_{t,0} - xbar)/gamma ; Eq. (3): x_{t+1,0} <- x_{t,0} - alpha gamma u
+    const float ue = __fmaf_rn(O.beta, comp(u0, e), __fmul_rn(__fsub_rn(comp(x0, e), comp(xbar, e)), O.inv_gamma));
+    comp(un, e) = ue;
+    comp(xn, e) = __fmaf_rn(O.neg_alpha_gamma, ue, comp(x0, e));
+  }
+  st_stream(O.u + col, un);
+  st_stream(O.anchor + col, xn);
+  store_rows(O.x + col, O.pitch, m, xn);
+  if (POLICY == 0) {
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    store_rows(O.h + col, O.pitch, m, zero);
+    if (BASE == 1) store_rows(O.v + col, O.pitch, m, zero);
+  } else if (POLICY == 2) {
+    store_rows(O.h + col, O.pitch, m, div4(sh, O.m_float));
+    if (BASE == 1) store_rows(O.v + col, O.pitch, m, div4(sv, O.m_float));
+  }
+}
+
+template <int BASE, int GRAD>
+inline void launch_last_step_outer_policy(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
+  const uint32_t blocks = (O.nvec + kThreads - 1) / kThreads;
+  constexpr int ROWS = BASE == 1 ? 2 : 4;
+  switch (policy) {
+    case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    default: last_step_outer_kernel<BASE, GRAD, 2, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
+  }
+}
+
+inline void launch_last_step_outer(const LocalArgs &L, const OuterArgs &O, bool adam, bool generated, int policy,
+                                   cudaStream_t stream) {
+  if (adam) {
+    if (generated) launch_last_step_outer_policy<1, 0>(L, O, policy, stream);
+    else launch_last_step_outer_policy<1, 1>(L, O, policy, stream);
+  } else {
+    if (generated) launch_last_step_outer_policy<0, 0>(L, O, policy, stream);
+    else launch_last_step_outer_policy<0, 1>(L, O, policy, stream);
+  }
+}
+
+}  // namespace slowmo

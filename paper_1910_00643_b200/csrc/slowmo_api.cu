@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "outer_fused.cuh"
 #include "outer_staged.cuh"
 
 using namespace slowmo;
@@ -28,6 +29,8 @@ struct slowmo_ctx {
   float gamma;               // gamma_t in force
   std::vector<uint64_t> tensor_offsets;  // n_tensors + 1 prefix sums, or empty
   int outer_variant;
+  bool pending_last;         // fused variant: the last inner step waits to run inside the outer step
+  LocalArgs pending;         // its arguments (counters k, l already include it)
   int *status_dev;           // device status block: [0] = timeout flag, [1] = where
   int cuda_error;
   int num_sms;
@@ -74,6 +77,24 @@ void launch_outer_direct(slowmo_ctx *ctx, const OuterArgs &A) {
   }
 }
 
+void launch_local_any(slowmo_ctx *ctx, const LocalArgs &A) {
+  const bool generated = ctx->cfg.grad_mode == SLOWMO_GRAD_GENERATED;
+  if (ctx->cfg.base == SLOWMO_BASE_NESTEROV) {
+    if (generated) launch_local<0, 0>(ctx, A); else launch_local<0, 1>(ctx, A);
+  } else {
+    if (generated) launch_local<1, 0>(ctx, A); else launch_local<1, 1>(ctx, A);
+  }
+}
+
+// Fused variant: run the deferred last inner step on its own (state is about to be read or
+// written from outside).
+int flush_pending(slowmo_ctx *ctx) {
+  if (!ctx->pending_last) return SLOWMO_OK;
+  ctx->pending_last = false;
+  launch_local_any(ctx, ctx->pending);
+  return check_launch(ctx);
+}
+
 // Resolve a tensor id to (base pointer, rows); NULL if the tensor does not exist here.
 float *tensor_base(slowmo_ctx *ctx, int which, uint32_t *rows) {
   const slowmo_buffers &b = ctx->buf;
@@ -99,6 +120,7 @@ int copy_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, ui
   if (replica < -1 || (replica >= 0 && (uint32_t)replica >= rows)) return SLOWMO_EINVAL;
   if (offset > ctx->cfg.P || count > ctx->cfg.P - offset) return SLOWMO_EINVAL;
   if (count == 0) return SLOWMO_OK;
+  if (int rc = flush_pending(ctx)) return rc;
   const uint32_t nrows = replica < 0 ? rows : 1;
   float *dev = base + (replica < 0 ? 0 : (uint64_t)replica * ctx->buf.pitch) + offset;
   const size_t width = count * sizeof(float), dpitch = ctx->buf.pitch * sizeof(float);
@@ -164,6 +186,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   ctx->pow_b1 = ctx->pow_b2 = 1.0;
   ctx->gamma = cfg->gamma;
   ctx->outer_variant = SLOWMO_VARIANT_DEFAULT;
+  ctx->pending_last = false;
   ctx->status_dev = nullptr;
   ctx->cuda_error = 0;
   if (cfg->n_tensors) {
@@ -228,6 +251,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
 
 int slowmo_destroy(slowmo_ctx *ctx) {
   if (!ctx) return SLOWMO_EINVAL;
+  flush_pending(ctx);
   cudaStreamSynchronize(ctx->stream);
   if (ctx->status_dev) cudaFree(ctx->status_dev);
   delete ctx;
@@ -274,12 +298,14 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     A.k = ctx->k;
     if (generated && c.m <= kInlineKeys)
       for (uint32_t i = 0; i < c.m; ++i) A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, i);
-    if (c.base == SLOWMO_BASE_NESTEROV) {
-      if (generated) launch_local<0, 0>(ctx, A); else launch_local<0, 1>(ctx, A);
-    } else {
-      if (generated) launch_local<1, 0>(ctx, A); else launch_local<1, 1>(ctx, A);
-    }
     ctx->k += 1;
+    // fused variant: step tau-1 is taken inside the outer-step kernel
+    if (ctx->outer_variant == SLOWMO_OUTER_FUSED && ctx->k == c.tau && (!generated || c.m <= kInlineKeys)) {
+      ctx->pending = A;
+      ctx->pending_last = true;
+      break;
+    }
+    launch_local_any(ctx, A);
     int rc = check_launch(ctx);
     if (rc != SLOWMO_OK) return rc;
   }
@@ -309,7 +335,14 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
 
   int variant = ctx->outer_variant;
   if (variant == SLOWMO_VARIANT_DEFAULT) variant = SLOWMO_OUTER_DIRECT;
-  if (variant == SLOWMO_OUTER_STAGED) {
+  if (ctx->pending_last && variant != SLOWMO_OUTER_FUSED) {
+    if (int rc = flush_pending(ctx)) return rc;
+  }
+  if (ctx->pending_last) {
+    ctx->pending_last = false;
+    launch_last_step_outer(ctx->pending, A, c.base == SLOWMO_BASE_ADAM, c.grad_mode == SLOWMO_GRAD_GENERATED,
+                           c.buffer_policy, ctx->stream);
+  } else if (variant == SLOWMO_OUTER_STAGED) {
     launch_outer_staged(A, nbuf, c.buffer_policy, ctx->num_sms, ctx->status_dev, ctx->stream);
   } else {
     if (nbuf == 1) launch_outer_direct<1>(ctx, A); else launch_outer_direct<2>(ctx, A);
@@ -386,8 +419,10 @@ int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_
 int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant) {
   if (!ctx) return SLOWMO_EINVAL;
   if (kernel == SLOWMO_K_OUTER) {
-    if (variant != SLOWMO_VARIANT_DEFAULT && variant != SLOWMO_OUTER_DIRECT && variant != SLOWMO_OUTER_STAGED)
+    if (variant != SLOWMO_VARIANT_DEFAULT && variant != SLOWMO_OUTER_DIRECT && variant != SLOWMO_OUTER_STAGED &&
+        variant != SLOWMO_OUTER_FUSED)
       return SLOWMO_EINVAL;
+    if (int rc = flush_pending(ctx)) return rc;
     ctx->outer_variant = variant;
     return SLOWMO_OK;
   }
@@ -398,6 +433,7 @@ int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant) {
 int slowmo_sync_status(slowmo_ctx *ctx) {
   if (!ctx) return SLOWMO_EINVAL;
   if (ctx->cuda_error) return SLOWMO_ECUDA;
+  if (int rc = flush_pending(ctx)) return rc;
   int host[4] = {0, 0, 0, 0};
   cudaError_t e = cudaMemcpyAsync(host, ctx->status_dev, sizeof(host), cudaMemcpyDeviceToHost, ctx->stream);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);

@@ -117,7 +117,7 @@ def test_product_code_never_touches_the_oracle():
 
 def test_workload_descriptions():
     from paper_1910_00643_b200 import workloads
-    from bench import local_step_bytes, outer_step_bytes
+    from bench import fused_outer_step_bytes, local_step_bytes, outer_step_bytes
     w = workloads.workload("resnet50")
     sizes = workloads.tensor_sizes(w["P"], w["n_tensors"], w["seed"])
     assert len(sizes) == 161 and int(sizes.sum()) == w["P"] and sizes.min() >= 1
@@ -134,6 +134,10 @@ def test_workload_descriptions():
     ws = workloads.workload("stress_tau12")
     assert local_step_bytes(ws) / (ws["m"] * ws["P"]) == 20
     assert outer_step_bytes(ws) / ws["P"] == 64
+    # outer step with the last inner step fused in: 20m + 16 (+4 for a) per parameter, +8m for Adam's v
+    assert fused_outer_step_bytes(ws) / ws["P"] == 96
+    assert fused_outer_step_bytes(w) / w["P"] == 20 * 32 + 20
+    assert fused_outer_step_bytes(wa) / wa["P"] == 28 * 8 + 20
     j = workloads.sample_coordinates(10**9, 1000, seed=1)
     assert j[0] == 0 and j[-1] == 10**9 - 1 and len(np.unique(j)) == len(j)
 

@@ -118,7 +118,7 @@ def test_supplied_gradient_fill_matches_oracle():
 SMALL_P = 3 * 1024 + 37  # several 512- and 1024-column tiles and a ragged tail (not a multiple of 4)
 
 
-@pytest.mark.parametrize("variant", ["direct", "staged"])
+@pytest.mark.parametrize("variant", ["direct", "staged", "fused"])
 @pytest.mark.parametrize("base,policy", list(itertools.product(("nesterov", "adam"), ("reset", "maintain", "average"))))
 @pytest.mark.parametrize("m", [1, 3, 4, 9])
 def test_small_runs_match_oracle(base, policy, m, variant):
@@ -137,7 +137,7 @@ def test_small_runs_match_oracle(base, policy, m, variant):
 @pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 511, 512, 513, 1023, 1024, 1025, 2048 + 4])
 def test_ragged_sizes(P):
     w = workloads.workload("tiny", P=P, m=5, tau=2, T=2, buffer_policy="average")
-    for variant in ("direct", "staged"):
+    for variant in ("direct", "staged", "fused"):
         s = _slowmo(w, guard=64)
         s.set_variant("outer", variant)
         s.run(2)
@@ -156,7 +156,7 @@ def test_tiny_workload_full_run():
 
 def test_many_workers():
     w = workloads.workload("tiny", P=2051, m=32, tau=2, T=2, buffer_policy="average")
-    for variant in ("direct", "staged"):
+    for variant in ("direct", "staged", "fused"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
@@ -190,7 +190,7 @@ def test_runs_are_bit_reproducible():
     import torch
     w = workloads.workload("resnet50", P=200_003, m=8, T=2, n_tensors=0)
     outs = []
-    for variant in ("direct", "staged", "direct"):
+    for variant in ("direct", "staged", "direct", "fused"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
@@ -200,6 +200,41 @@ def test_runs_are_bit_reproducible():
     for other in outs[1:]:
         for a, b in zip(outs[0], other):
             assert torch.equal(a, b)
+
+
+def test_fused_last_step_is_transparent_through_the_api():
+    # the deferred last inner step must be invisible: reading state between the inner loop and
+    # the outer step runs it, and the run still ends bit-identical to the oracle
+    w = workloads.workload("tiny", P=3000, m=3, tau=3, T=2, buffer_policy="maintain")
+    ref_mid = oracle.run(oracle.make_config(**dict(w, T=1, alpha=1.0, beta=0.0)), j0=0, n=w["P"])
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", "fused")
+    s.local_steps(3)
+    h_mid = s.get_params("h")            # forces the deferred step; h after tau steps of iteration 0
+    assert np.array_equal(h_mid.view(np.uint32), ref_mid["h"].view(np.uint32))
+    s.outer_step()
+    s.local_steps(2)
+    s.local_steps(1)                     # deferred again, taken inside the outer-step kernel
+    s.outer_step()
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+    # tau = 1: every inner step is the last one
+    w1 = workloads.workload("sync_sgd", P=2500, m=4, T=3)
+    s = _slowmo(w1)
+    s.set_variant("outer", "fused")
+    s.run(3)
+    _check_against_oracle(s, w1, np.arange(w1["P"]), exact=True)
+    s.close()
+    # supplied gradient
+    w2 = workloads.workload("stress_tau12", P=4100, m=4, tau=2, T=2)
+    s = _slowmo(w2)
+    s.set_variant("outer", "fused")
+    s.alloc_gradient()
+    s.fill_gradient()
+    s.run(2, s.grad)
+    _check_against_oracle(s, w2, np.arange(w2["P"]), exact=True)
+    s.close()
 
 
 def test_learning_rate_schedule():
@@ -376,11 +411,11 @@ def test_full_size_supplied_gradient_on_sampled_coordinates(name):
     torch.cuda.empty_cache()
 
 
-def test_full_size_staged_outer_step_equals_direct():
+def test_full_size_staged_and_fused_outer_steps_equal_direct():
     import torch
     w = workloads.workload("resnet50", T=2)
     res = []
-    for variant in ("direct", "staged"):
+    for variant in ("direct", "staged", "fused"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
@@ -390,5 +425,6 @@ def test_full_size_staged_outer_step_equals_direct():
         s.close()
         del s
         torch.cuda.empty_cache()
-    for a, b in zip(*res):
-        assert torch.equal(a[..., :w["P"]], b[..., :w["P"]])
+    for other in res[1:]:
+        for a, b in zip(res[0], other):
+            assert torch.equal(a[..., :w["P"]], b[..., :w["P"]])
