@@ -10,7 +10,7 @@ import numpy as np
 
 from . import build as _build
 
-BASE = {"nesterov": 0, "adam": 1}
+BASE = {"nesterov": 0, "adam": 1, "sgp_nesterov": 2, "sgp_adam": 3}
 POLICY = {"reset": 0, "maintain": 1, "average": 2}
 GRAD = {"generated": 0, "supplied_hash": 1, "supplied": 1, "supplied_array": 2}
 TAG_CURVATURE, TAG_CENTRE, TAG_GRADNOISE, TAG_SUPPLIED = 1, 2, 3, 5
@@ -61,6 +61,8 @@ def lib():
         L.oracle_centre.argtypes = [C.POINTER(_Cfg), C.c_uint32, C.c_uint64]
         L.oracle_supplied_gradient.argtypes = [C.POINTER(_Cfg), C.c_uint32, C.c_uint64]
         L.slowmo_oracle_threads.restype = C.c_int
+        L.oracle_sgp_hops.restype = C.c_uint32
+        L.oracle_sgp_hops.argtypes = [C.c_uint32, C.c_uint64]
         _lib = L
     return _lib
 
@@ -140,6 +142,11 @@ def centre(cfg, w, j):
 
 def supplied_gradient(cfg, w, j):
     return np.array([lib().oracle_supplied_gradient(C.byref(cfg), w, int(q)) for q in j], np.float32)
+
+
+def sgp_hops(m, s):
+    """Hop distance of the directed exponential graph at global step s."""
+    return lib().oracle_sgp_hops(m, s)
 
 
 def threads():

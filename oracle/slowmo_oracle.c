@@ -13,6 +13,13 @@
  *  - Weight decay is L2: added to the gradient before the momentum update.
  *  - The buffer policy of outer iteration t+1 is applied right after the outer update
  *    of iteration t (at t = 0 every policy is a no-op because the buffers are zero).
+ *  - Stochastic gradient push (Algorithm 2; Table C.1, SGP rows): the graph is the
+ *    time-varying directed exponential graph with one peer per step: at global step
+ *    s = t tau + k worker i sends to worker (i + 2^q) mod m, q = s mod (floor(log2(m-1)) + 1),
+ *    and keeps half: p^(i,i) = p^(i+2^q,i) = 1/2. The push-sum weights w start at 1 and are
+ *    set back to 1 after each outer step (all workers then hold the same model). The
+ *    gradient (and the L2 term) is taken at the de-biased z = x / w; the exact average of
+ *    Algorithm 1 is over x.
  *  - 1/gamma_t and alpha*gamma_t are formed once per outer iteration (in binary64,
  *    rounded once to `real`); the worker sum runs in worker order 0..m-1 and is divided
  *    by m.
@@ -55,9 +62,18 @@ static real gradient(const oracle_config *cfg, uint32_t i, uint64_t j, uint32_t 
   return g;
 }
 
+#if !ORACLE_F64
+uint32_t oracle_sgp_hops(uint32_t m, uint64_t s) {
+  if (m < 2) return 0;
+  uint32_t nq = 0; /* floor(log2(m-1)) + 1 */
+  for (uint32_t r = m - 1; r > 0; r >>= 1) nq += 1;
+  return 1u << (uint32_t)(s % nq);
+}
+#endif
+
 static int valid(const oracle_config *c) {
   if (c->m == 0 || c->tau == 0) return 0;
-  if (c->base != ORACLE_BASE_NESTEROV && c->base != ORACLE_BASE_ADAM) return 0;
+  if (c->base < ORACLE_BASE_NESTEROV || c->base > ORACLE_BASE_SGP_ADAM) return 0;
   if (c->buffer_policy < ORACLE_BUF_RESET || c->buffer_policy > ORACLE_BUF_AVERAGE) return 0;
   if (c->grad_mode < ORACLE_GRAD_GENERATED || c->grad_mode > ORACLE_GRAD_SUPPLIED_ARRAY) return 0;
   return 1;
@@ -69,7 +85,8 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
   if (!cfg || !valid(cfg) || !x_out || !anchor_out || !u_out || !h_out) return -1;
   if (cfg->grad_mode == ORACLE_GRAD_SUPPLIED_ARRAY && !G) return -1;
   const uint32_t m = cfg->m, tau = cfg->tau, T = cfg->T;
-  const int adam = cfg->base == ORACLE_BASE_ADAM;
+  const int adam = cfg->base == ORACLE_BASE_ADAM || cfg->base == ORACLE_BASE_SGP_ADAM;
+  const int sgp = cfg->base == ORACLE_BASE_SGP_NESTEROV || cfg->base == ORACLE_BASE_SGP_ADAM;
   const real mu = (real)cfg->mu;
   const real b1 = (real)cfg->adam_b1, b2 = (real)cfg->adam_b2, eps = (real)cfg->adam_eps;
   const real omb1 = (real)(1.0 - (double)cfg->adam_b1); /* 1 - beta_1 */
@@ -84,6 +101,9 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
     real *v = (real *)malloc(sizeof(real) * m);
     real *c = (real *)malloc(sizeof(real) * m);
     real *Gfix = (real *)malloc(sizeof(real) * m);
+    real *w = (real *)malloc(sizeof(real) * m);     /* push-sum weights w^{(i)}      */
+    real *x_half = (real *)malloc(sizeof(real) * m); /* x_{k+1/2}^{(i)} of Algorithm 2 */
+    real *w_half = (real *)malloc(sizeof(real) * m);
 
 #pragma omp for schedule(static)
     for (uint64_t q = 0; q < n; ++q) {
@@ -106,6 +126,7 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
         x[i] = x0;
         h[i] = 0;
         v[i] = 0;
+        w[i] = 1;
       }
       uint64_t l = 0;            /* Adam steps since the buffers were last zero */
       double pow_b1 = 1.0, pow_b2 = 1.0; /* beta_1^l, beta_2^l */
@@ -128,7 +149,9 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
             real G_ij = Gfix[i];
             if (cfg->grad_mode == ORACLE_GRAD_SUPPLIED_ARRAY)
               G_ij = (real)G[(((uint64_t)t * tau + k) * m + i) * n + q];
-            const real g = gradient(cfg, i, j, t, k, x[i], a_j, c[i], G_ij);
+            /* SGP evaluates the gradient at the de-biased parameters z = x / w */
+            const real at = sgp ? x[i] / w[i] : x[i];
+            const real g = gradient(cfg, i, j, t, k, at, a_j, c[i], G_ij);
             real d;
             if (!adam) {
               /* Table C.1, SGD row: h <- mu h + g ; d = mu h + g (Nesterov momentum) */
@@ -147,6 +170,21 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
             dsum += (double)d;
           }
           if (dbar) dbar[((uint64_t)t * tau + k) * n + q] = dsum / (double)m;
+
+          if (sgp && m > 1) {
+            /* Algorithm 2: the step above gave x_{k+1/2}; every worker keeps half of
+             * (x_{k+1/2}, w) and receives half of its in-neighbour's */
+            const uint32_t hops = oracle_sgp_hops(m, (uint64_t)t * tau + k);
+            for (uint32_t i = 0; i < m; ++i) {
+              x_half[i] = x[i];
+              w_half[i] = w[i];
+            }
+            for (uint32_t i = 0; i < m; ++i) {
+              const uint32_t from = (i + m - hops % m) % m; /* the worker that sends to i */
+              x[i] = (real)0.5 * x_half[i] + (real)0.5 * x_half[from];
+              w[i] = (real)0.5 * w_half[i] + (real)0.5 * w_half[from];
+            }
+          }
         }
 
         /* Algorithm 1, exact average over the workers */
@@ -158,7 +196,10 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
         /* Eq. (3): x_{t+1,0} = x_{t,0} - alpha gamma_t u_{t+1} */
         x0 = FMA(-alpha_gam, u, x0);
         /* every worker continues from x_{t+1,0} */
-        for (uint32_t i = 0; i < m; ++i) x[i] = x0;
+        for (uint32_t i = 0; i < m; ++i) {
+          x[i] = x0;
+          w[i] = 1;
+        }
 
         /* buffer policy for the next outer iteration */
         if (cfg->buffer_policy == ORACLE_BUF_RESET) {
@@ -192,6 +233,9 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
     free(v);
     free(c);
     free(Gfix);
+    free(w);
+    free(x_half);
+    free(w_half);
   }
   return 0;
 }

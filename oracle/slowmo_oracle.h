@@ -57,7 +57,12 @@ void oracle_stream_export(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, u
 
 /* ---- Algorithm 1 (slowmo_oracle.c) -------------------------------------------------- */
 
-enum { ORACLE_BASE_NESTEROV = 0, ORACLE_BASE_ADAM = 1 };
+enum {
+  ORACLE_BASE_NESTEROV = 0,     /* Table C.1, SGD row (local Nesterov momentum, no communication) */
+  ORACLE_BASE_ADAM = 1,         /* Table C.1, Adam row                                             */
+  ORACLE_BASE_SGP_NESTEROV = 2, /* Algorithm 2 (stochastic gradient push with Nesterov momentum)   */
+  ORACLE_BASE_SGP_ADAM = 3      /* Table C.1, SGP (Adam) row                                       */
+};
 enum { ORACLE_BUF_RESET = 0, ORACLE_BUF_MAINTAIN = 1, ORACLE_BUF_AVERAGE = 2 };
 enum {
   ORACLE_GRAD_GENERATED = 0,     /* noisy quadratic gradient, generated from the hash     */
@@ -103,6 +108,10 @@ int slowmo_oracle_run_f32(const oracle_config *cfg, const float *gamma_t, const 
 int slowmo_oracle_run_f64(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_idx,
                           uint64_t j0, uint64_t n, const float *G, double *x, double *anchor,
                           double *u, double *h, double *v, double *dbar);
+
+/* Hop distance 2^q of the directed exponential graph at global base-optimizer step s for m
+ * workers: q cycles through 0 .. floor(log2(m-1)); 0 when m = 1 (no peer). */
+uint32_t oracle_sgp_hops(uint32_t m, uint64_t s);
 
 /* Synthetic inputs for coordinates, as the run above sees them (fp32 values). */
 float oracle_curvature(const oracle_config *cfg, uint64_t j);
