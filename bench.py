@@ -40,7 +40,7 @@ def local_step_bytes(w):
     """Algorithmic HBM bytes of one fused local-step launch: x and h (and v) read and written,
     the per-worker gradient data (centres c, or the supplied gradient) read, and the curvature
     read once for all workers."""
-    per_update = 8 + 8 + 4 + (8 if w["base"] == "adam" else 0)
+    per_update = 8 + 8 + 4 + (8 if "adam" in w["base"] else 0)
     total = per_update * w["m"] * w["P"]
     if w["grad_mode"] == "generated":
         total += 4 * w["P"]
@@ -52,7 +52,7 @@ def outer_step_bytes(w):
     and u read and written, plus the buffer policy (reset: nb*m rows written; average: nb*m
     rows read and written)."""
     m, P = w["m"], w["P"]
-    nb = 2 if w["base"] == "adam" else 1
+    nb = 2 if "adam" in w["base"] else 1
     per_param = 8 * m + 16
     if w["buffer_policy"] == "reset":
         per_param += 4 * m * nb
@@ -67,7 +67,7 @@ def fused_outer_step_bytes(w):
     the m rows of x written; the m rows of h [, v] written once under every policy (stepped
     values, zeros or means)."""
     m, P = w["m"], w["P"]
-    nb = 2 if w["base"] == "adam" else 1
+    nb = 2 if "adam" in w["base"] else 1
     per_param = m * (4 + 4 * nb + 4) + 8 + 8 + m * 4 + m * 4 * nb
     if w["grad_mode"] == "generated":
         per_param += 4
@@ -318,7 +318,8 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     s = SlowMo(w)
     s.set_variant("outer", args.outer_variant)
-    fused = args.outer_variant == "fused" and (w["grad_mode"] == "supplied" or w["m"] <= 64) and w["tau"] > 1
+    fused = (args.outer_variant == "fused" and (w["grad_mode"] == "supplied" or w["m"] <= 64) and w["tau"] > 1
+             and not w["base"].startswith("sgp"))
     grad = None
     if w["grad_mode"] == "supplied":
         grad = s.alloc_gradient()

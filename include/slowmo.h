@@ -50,7 +50,12 @@ enum {
   SLOWMO_ETIMEOUT = -6, /* a bounded device-side wait gave up                       */
   SLOWMO_ENOTIMPL = -7
 };
-enum { SLOWMO_BASE_NESTEROV = 0, SLOWMO_BASE_ADAM = 1 };
+enum {
+  SLOWMO_BASE_NESTEROV = 0,     /* Table C.1, SGD row: local Nesterov momentum, no communication   */
+  SLOWMO_BASE_ADAM = 1,         /* Table C.1, Adam row                                              */
+  SLOWMO_BASE_SGP_NESTEROV = 2, /* Algorithm 2: stochastic gradient push with Nesterov momentum     */
+  SLOWMO_BASE_SGP_ADAM = 3      /* Table C.1, SGP (Adam) row                                        */
+};
 enum { SLOWMO_BUF_RESET = 0, SLOWMO_BUF_MAINTAIN = 1, SLOWMO_BUF_AVERAGE = 2 };
 enum { SLOWMO_GRAD_GENERATED = 0, SLOWMO_GRAD_SUPPLIED = 1 };
 /* tensors addressable by slowmo_get_params / slowmo_set_params */
@@ -141,6 +146,16 @@ int slowmo_destroy(slowmo_ctx *ctx);
  *              l = Adam steps since the buffers were last zero (1-based)
  *   step       x = fma(-gamma_t, d, x)                                     (Algorithm 1)
  *
+ *   SGP bases  the step above yields x_{k+1/2}; then the push-sum mixing of Algorithm 2 on the
+ *              time-varying directed exponential graph, one peer per step: with
+ *              hops = 2^q, q = (t*tau + k) mod (floor(log2(m-1)) + 1), worker i keeps half and
+ *              receives half from worker (i - hops) mod m:
+ *              x_i = 0.5*x_{k+1/2,i} + 0.5*x_{k+1/2,(i-hops) mod m}.
+ *              This mixing matrix is doubly stochastic, so the push-sum weights stay exactly 1
+ *              and the de-biased z equals x; the gradient is therefore evaluated at x.
+ *              SGP bases need m <= 64 (ENOTIMPL from slowmo_create otherwise) and ignore
+ *              SLOWMO_OUTER_FUSED.
+ *
  * `grad` is a device [m, pitch] tensor in supplied mode (read by each of the n steps) and
  * must be NULL in generated mode (EINVAL otherwise).
  *
@@ -230,8 +245,8 @@ int slowmo_sync_status(slowmo_ctx *ctx);
  * Computes exactly what slowmo_outer_step computes (same kernel, same arithmetic, same
  * order): average of the m rows of x, Eq. (2), Eq. (3), broadcast, buffer policy, on the
  * caller's device tensors x, h [m, pitch], v [m, pitch] (Adam only, else NULL), anchor,
- * u [pitch], with the layout rules at the top of this file. base and buffer_policy are
- * SLOWMO_BASE_* / SLOWMO_BUF_* (base only tells whether v exists).
+ * u [pitch], with the layout rules at the top of this file. base is SLOWMO_BASE_NESTEROV or
+ * SLOWMO_BASE_ADAM (it only tells whether v exists); buffer_policy is SLOWMO_BUF_*.
  *
  * Limits: the scratch does not grow with the problem, so the only size limits are the
  * kernel's index range: 1 <= P <= SLOWMO_STATIC_MAX_P and 1 <= m <= SLOWMO_STATIC_MAX_M;

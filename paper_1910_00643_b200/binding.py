@@ -14,7 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libslowmo.so")
 
 OK, EINVAL, ESTATE, EALIGN, ECUDA, ENOMEM, ETIMEOUT, ENOTIMPL = 0, -1, -2, -3, -4, -5, -6, -7
-BASE = {"nesterov": 0, "adam": 1}
+BASE = {"nesterov": 0, "adam": 1, "sgp_nesterov": 2, "sgp_adam": 3}
 POLICY = {"reset": 0, "maintain": 1, "average": 2}
 GRAD = {"generated": 0, "supplied": 1}
 TENSOR = {"x": 0, "anchor": 1, "u": 2, "h": 3, "v": 4, "a": 5, "c": 6}
@@ -157,7 +157,7 @@ class SlowMo:
         self.pitch = pitch if pitch is not None else round_up(self.P, 32)
         self.stream = stream if stream is not None else torch.cuda.Stream()
         self.guard = guard
-        adam = self.cfg.base == BASE["adam"]
+        adam = self.cfg.base in (BASE["adam"], BASE["sgp_adam"])
         generated = self.cfg.grad_mode == GRAD["generated"]
         self._raw = {}
         self.t = {}

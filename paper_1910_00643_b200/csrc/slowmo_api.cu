@@ -14,6 +14,7 @@
 #include "kernels.cuh"
 #include "outer_fused.cuh"
 #include "outer_staged.cuh"
+#include "sgp_step.cuh"
 
 using namespace slowmo;
 
@@ -38,6 +39,8 @@ struct slowmo_ctx {
 
 namespace {
 
+bool is_adam(int base) { return base == SLOWMO_BASE_ADAM || base == SLOWMO_BASE_SGP_ADAM; }
+bool is_sgp(int base) { return base == SLOWMO_BASE_SGP_NESTEROV || base == SLOWMO_BASE_SGP_ADAM; }
 bool finite_pos(float v) { return std::isfinite(v) && v > 0.0f; }
 bool unit_interval(float v) { return std::isfinite(v) && v >= 0.0f && v < 1.0f; }
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -79,7 +82,10 @@ void launch_outer_direct(slowmo_ctx *ctx, const OuterArgs &A) {
 
 void launch_local_any(slowmo_ctx *ctx, const LocalArgs &A) {
   const bool generated = ctx->cfg.grad_mode == SLOWMO_GRAD_GENERATED;
-  if (ctx->cfg.base == SLOWMO_BASE_NESTEROV) {
+  if (is_sgp(ctx->cfg.base)) {
+    // Algorithm 2: the graph's hop distance follows the global step count t*tau + k
+    launch_sgp_step(A, sgp_hops(A.m, A.t * ctx->cfg.tau + A.k), is_adam(ctx->cfg.base), generated, ctx->stream);
+  } else if (ctx->cfg.base == SLOWMO_BASE_NESTEROV) {
     if (generated) launch_local<0, 0>(ctx, A); else launch_local<0, 1>(ctx, A);
   } else {
     if (generated) launch_local<1, 0>(ctx, A); else launch_local<1, 1>(ctx, A);
@@ -144,12 +150,13 @@ extern "C" {
 int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cuda_stream, slowmo_ctx **out) {
   if (!cfg || !buf || !out) return SLOWMO_EINVAL;
   *out = nullptr;
-  const bool adam = cfg->base == SLOWMO_BASE_ADAM;
+  const bool adam = is_adam(cfg->base);
   const bool generated = cfg->grad_mode == SLOWMO_GRAD_GENERATED;
   if (cfg->P == 0 || cfg->m == 0 || cfg->tau == 0) return SLOWMO_EINVAL;
+  if (cfg->base < SLOWMO_BASE_NESTEROV || cfg->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
+  if (is_sgp(cfg->base) && cfg->m > kSgpMaxWorkers) return SLOWMO_ENOTIMPL;
   if (cfg->P > (1ull << 32) - 4096) return SLOWMO_EINVAL;  // columns are indexed with 32 bits
   if (!finite_pos(cfg->alpha) || !unit_interval(cfg->beta) || !finite_pos(cfg->gamma)) return SLOWMO_EINVAL;
-  if (cfg->base != SLOWMO_BASE_NESTEROV && !adam) return SLOWMO_EINVAL;
   if (cfg->buffer_policy < SLOWMO_BUF_RESET || cfg->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
   if (!generated && cfg->grad_mode != SLOWMO_GRAD_SUPPLIED) return SLOWMO_EINVAL;
   if (!std::isfinite(cfg->weight_decay) || cfg->weight_decay < 0.0f || !std::isfinite(cfg->x_init)) return SLOWMO_EINVAL;
@@ -218,6 +225,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   if (e == cudaSuccess) e = cudaMalloc(&ctx->status_dev, 4 * sizeof(int));
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status_dev, 0, 4 * sizeof(int), ctx->stream);
   if (e == cudaSuccess) e = outer_staged_configure();
+  if (e == cudaSuccess && is_sgp(cfg->base)) e = sgp_configure();
   if (e != cudaSuccess) {
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     delete ctx;
@@ -300,7 +308,8 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
       for (uint32_t i = 0; i < c.m; ++i) A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, i);
     ctx->k += 1;
     // fused variant: step tau-1 is taken inside the outer-step kernel
-    if (ctx->outer_variant == SLOWMO_OUTER_FUSED && ctx->k == c.tau && (!generated || c.m <= kInlineKeys)) {
+    if (ctx->outer_variant == SLOWMO_OUTER_FUSED && ctx->k == c.tau && (!generated || c.m <= kInlineKeys) &&
+        !is_sgp(c.base)) {
       ctx->pending = A;
       ctx->pending_last = true;
       break;
@@ -331,7 +340,7 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
   A.inv_gamma = (float)(1.0 / (double)ctx->gamma);
   A.neg_alpha_gamma = -(float)((double)c.alpha * (double)ctx->gamma);
   A.m_float = (float)c.m;
-  const int nbuf = c.base == SLOWMO_BASE_ADAM ? 2 : 1;
+  const int nbuf = is_adam(c.base) ? 2 : 1;
 
   int variant = ctx->outer_variant;
   if (variant == SLOWMO_VARIANT_DEFAULT) variant = SLOWMO_OUTER_DIRECT;

@@ -44,6 +44,15 @@ WORKLOADS = {
                              gamma=5e-4, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8,
                              weight_decay=0.0, a_lo=0.1, a_hi=1.0, c_std=0.02, sigma=0.01,
                              seed=0, x_init=0.0),
+    # stochastic gradient push as the base optimizer (the paper's SGP + SlowMo on ImageNet: tau = 48,
+    # Nesterov buffers zeroed at each outer step) and its Adam form (WMT'16)
+    "sgp_resnet50": dict(P=25_557_032, m=32, tau=48, T=3, alpha=1.0, beta=0.6, buffer_policy="reset",
+                         grad_mode="generated", base="sgp_nesterov", gamma=0.1, mu=0.9, weight_decay=1e-4,
+                         a_lo=0.1, a_hi=1.0, c_std=0.05, sigma=0.01, seed=0, x_init=0.0),
+    "sgp_transformer_adam": dict(P=210_000_000, m=8, tau=48, T=2, alpha=1.0, beta=0.5,
+                                 buffer_policy="maintain", grad_mode="generated", base="sgp_adam",
+                                 gamma=5e-4, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8, weight_decay=0.0,
+                                 a_lo=0.1, a_hi=1.0, c_std=0.02, sigma=0.01, seed=0, x_init=0.0),
     # bandwidth stress: supplied gradient tensor, tau swept over {1, 12, 48}
     "stress_tau1": dict(P=1_000_000_000, m=4, tau=1, T=3, alpha=1.0, beta=0.6,
                         buffer_policy="reset", grad_mode="supplied", sigma=0.1, seed=0,

@@ -24,7 +24,7 @@ def _slowmo(w, **kw):
 
 
 def _state_keys(w):
-    return ("x", "anchor", "u", "h") + (("v",) if w.get("base") == "adam" else ())
+    return ("x", "anchor", "u", "h") + (("v",) if "adam" in w.get("base", "") else ())
 
 
 def _gather(s, key, j):
@@ -278,6 +278,57 @@ def test_supplied_hash_gradient_small():
     _check_against_oracle(s, w, np.arange(5000), exact=True)
     assert s.guards_intact()
     s.close()
+
+
+# ------------------------------------------------------------------ stochastic gradient push bases
+
+@pytest.mark.parametrize("base,policy", [("sgp_nesterov", "reset"), ("sgp_nesterov", "average"),
+                                         ("sgp_adam", "maintain"), ("sgp_adam", "reset")])
+@pytest.mark.parametrize("m", [1, 2, 3, 8, 13, 32, 50, 64])
+def test_sgp_small_runs_match_oracle(base, policy, m):
+    w = workloads.workload("tiny", P=2 * 1024 + 37, m=m, tau=5, T=2, base=base, buffer_policy=policy, alpha=0.9,
+                           beta=0.6, gamma=0.01 if "adam" in base else 0.05, weight_decay=1e-3, adam_b1=0.9,
+                           adam_b2=0.98, adam_eps=1e-8, seed=9)
+    s = _slowmo(w, guard=64)
+    s.run(w["T"])
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+
+
+def test_sgp_supplied_gradient_and_step_by_step_calls():
+    w = workloads.workload("stress_tau12", P=3000, m=5, tau=7, T=2, base="sgp_nesterov")
+    s = _slowmo(w)
+    s.alloc_gradient()
+    s.fill_gradient()
+    for _ in range(2):
+        for n in (3, 1, 3):        # the graph position must follow the global step count across calls
+            s.local_steps(n, s.grad)
+        s.outer_step()
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    s.close()
+
+
+def test_sgp_needs_at_most_64_workers():
+    from paper_1910_00643_b200 import SlowMoError, binding
+    with pytest.raises(SlowMoError) as e:
+        _slowmo(workloads.workload("tiny", m=65, base="sgp_nesterov"))
+    assert e.value.status == binding.ENOTIMPL
+
+
+@pytest.mark.parametrize("name", ["sgp_resnet50", "sgp_transformer_adam"])
+def test_full_size_sgp_workloads_on_sampled_coordinates(name):
+    import torch
+    w = workloads.workload(name)
+    s = _slowmo(w)
+    s.run(w["T"])
+    j = workloads.sample_coordinates(w["P"], 1 << 12, seed=3)
+    _check_against_oracle(s, w, j, exact=True)
+    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
+    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    s.close()
+    del s
+    torch.cuda.empty_cache()
 
 
 # --------------------------------------------------------------------------- boundary behaviour
