@@ -25,7 +25,7 @@ class _Cfg(C.Structure):
         ("buffer_policy", C.c_int32), ("grad_mode", C.c_int32),
         ("seed", C.c_uint64),
         ("a_lo", C.c_float), ("a_hi", C.c_float), ("c_std", C.c_float), ("sigma", C.c_float),
-        ("x_init", C.c_float),
+        ("x_init", C.c_float), ("no_average", C.c_int32),
     ]
 
 
@@ -70,11 +70,11 @@ def lib():
 def make_config(*, m, tau, T, alpha=1.0, beta=0.0, gamma=0.1, base="nesterov", mu=0.0,
                 weight_decay=0.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8,
                 buffer_policy="reset", grad_mode="generated", seed=0, a_lo=0.5, a_hi=2.0,
-                c_std=1.0, sigma=0.0, x_init=0.0, **_ignored):
+                c_std=1.0, sigma=0.0, x_init=0.0, no_average=False, **_ignored):
     """Build the C config. Names follow Algorithm 1 / Table C.1 of the paper."""
     return _Cfg(m, tau, T, alpha, beta, gamma, BASE[base], mu, weight_decay, adam_b1, adam_b2,
                 adam_eps, POLICY[buffer_policy], GRAD[grad_mode], seed, a_lo, a_hi, c_std, sigma,
-                x_init)
+                x_init, 1 if no_average else 0)
 
 
 def _ptr(a):
@@ -97,7 +97,8 @@ def run(cfg, *, j=None, j0=0, n=None, precision="f32", gamma_t=None, G=None, wan
     m = cfg.m
     out = {
         "x": np.empty((m, n), dt), "h": np.empty((m, n), dt), "v": np.empty((m, n), dt),
-        "anchor": np.empty(n, dt), "u": np.empty(n, dt),
+        "anchor": np.empty((m, n) if cfg.no_average else n, dt),
+        "u": np.empty((m, n) if cfg.no_average else n, dt),
     }
     dbar = np.empty((cfg.T, cfg.tau, n), np.float64) if want_dbar else None
     if gamma_t is not None:

@@ -20,6 +20,10 @@
  *    set back to 1 after each outer step (all workers then hold the same model). The
  *    gradient (and the L2 term) is taken at the de-biased z = x / w; the exact average of
  *    Algorithm 1 is over x.
+ *  - Section 6's variant without the exact average (no_average): each worker keeps its own
+ *    outer iterate x_{t,0}^{(i)} and slow momentum u^{(i)} and applies Eq. (2), (3) with its
+ *    own x_{t,tau}^{(i)} in place of the average; the buffer policy "average" would need the
+ *    communication the variant removes and is rejected. Push-sum weights are left alone.
  *  - 1/gamma_t and alpha*gamma_t are formed once per outer iteration (in binary64,
  *    rounded once to `real`); the worker sum runs in worker order 0..m-1 and is divided
  *    by m.
@@ -76,6 +80,7 @@ static int valid(const oracle_config *c) {
   if (c->base < ORACLE_BASE_NESTEROV || c->base > ORACLE_BASE_SGP_ADAM) return 0;
   if (c->buffer_policy < ORACLE_BUF_RESET || c->buffer_policy > ORACLE_BUF_AVERAGE) return 0;
   if (c->grad_mode < ORACLE_GRAD_GENERATED || c->grad_mode > ORACLE_GRAD_SUPPLIED_ARRAY) return 0;
+  if (c->no_average && c->buffer_policy == ORACLE_BUF_AVERAGE) return 0;
   return 1;
 }
 
@@ -104,6 +109,8 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
     real *w = (real *)malloc(sizeof(real) * m);     /* push-sum weights w^{(i)}      */
     real *x_half = (real *)malloc(sizeof(real) * m); /* x_{k+1/2}^{(i)} of Algorithm 2 */
     real *w_half = (real *)malloc(sizeof(real) * m);
+    real *x0_own = (real *)malloc(sizeof(real) * m); /* no_average: x_{t,0}^{(i)} */
+    real *u_own = (real *)malloc(sizeof(real) * m);  /* no_average: u^{(i)}       */
 
 #pragma omp for schedule(static)
     for (uint64_t q = 0; q < n; ++q) {
@@ -127,6 +134,8 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
         h[i] = 0;
         v[i] = 0;
         w[i] = 1;
+        x0_own[i] = x0;
+        u_own[i] = 0;
       }
       uint64_t l = 0;            /* Adam steps since the buffers were last zero */
       double pow_b1 = 1.0, pow_b2 = 1.0; /* beta_1^l, beta_2^l */
@@ -187,18 +196,27 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
           }
         }
 
-        /* Algorithm 1, exact average over the workers */
-        real s = x[0];
-        for (uint32_t i = 1; i < m; ++i) s = s + x[i];
-        const real xbar = s / (real)m;
-        /* Eq. (2): u_{t+1} = beta u_t + (x_{t,0} - xbar_{t,tau}) / gamma_t */
-        u = FMA(beta, u, (x0 - xbar) * inv_gam);
-        /* Eq. (3): x_{t+1,0} = x_{t,0} - alpha gamma_t u_{t+1} */
-        x0 = FMA(-alpha_gam, u, x0);
-        /* every worker continues from x_{t+1,0} */
-        for (uint32_t i = 0; i < m; ++i) {
-          x[i] = x0;
-          w[i] = 1;
+        if (!cfg->no_average) {
+          /* Algorithm 1, exact average over the workers */
+          real s = x[0];
+          for (uint32_t i = 1; i < m; ++i) s = s + x[i];
+          const real xbar = s / (real)m;
+          /* Eq. (2): u_{t+1} = beta u_t + (x_{t,0} - xbar_{t,tau}) / gamma_t */
+          u = FMA(beta, u, (x0 - xbar) * inv_gam);
+          /* Eq. (3): x_{t+1,0} = x_{t,0} - alpha gamma_t u_{t+1} */
+          x0 = FMA(-alpha_gam, u, x0);
+          /* every worker continues from x_{t+1,0} */
+          for (uint32_t i = 0; i < m; ++i) {
+            x[i] = x0;
+            w[i] = 1;
+          }
+        } else {
+          /* Section 6: the same two updates per worker, on its own x_{t,tau}^{(i)} */
+          for (uint32_t i = 0; i < m; ++i) {
+            u_own[i] = FMA(beta, u_own[i], (x0_own[i] - x[i]) * inv_gam);
+            x0_own[i] = FMA(-alpha_gam, u_own[i], x0_own[i]);
+            x[i] = x0_own[i];
+          }
         }
 
         /* buffer policy for the next outer iteration */
@@ -225,8 +243,15 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
         h_out[(uint64_t)i * n + q] = h[i];
         if (v_out) v_out[(uint64_t)i * n + q] = v[i];
       }
-      anchor_out[q] = x0;
-      u_out[q] = u;
+      if (!cfg->no_average) {
+        anchor_out[q] = x0;
+        u_out[q] = u;
+      } else {
+        for (uint32_t i = 0; i < m; ++i) {
+          anchor_out[(uint64_t)i * n + q] = x0_own[i];
+          u_out[(uint64_t)i * n + q] = u_own[i];
+        }
+      }
     }
     free(x);
     free(h);
@@ -236,6 +261,8 @@ int RUN_NAME(const oracle_config *cfg, const float *gamma_t, const uint64_t *j_i
     free(w);
     free(x_half);
     free(w_half);
+    free(x0_own);
+    free(u_own);
   }
   return 0;
 }

@@ -88,6 +88,9 @@ typedef struct {
   float c_std;           /* centre c_{w,j} ~ N(0, c_std^2)   */
   float sigma;           /* gradient-noise scale             */
   float x_init;          /* x_{0,0} in every coordinate      */
+  int32_t no_average;    /* 0: Algorithm 1 as printed. 1: the variant of Section 6 that skips the
+                            exact average: every worker applies Eq. (2), (3) to its own x_{t,tau},
+                            with its own slow momentum u^{(i)} and its own outer iterate           */
 } oracle_config;
 
 /*
@@ -96,7 +99,7 @@ typedef struct {
  *   gamma_t   NULL, or T base learning rates, one per outer iteration.
  *   G         only for ORACLE_GRAD_SUPPLIED_ARRAY: [T*tau][m][n] gradients, step-major.
  *   x, h, v   outputs [m][n] (row = worker); v may be NULL for Nesterov.
- *   anchor,u  outputs [n]: x_{T,0} and u_T.
+ *   anchor,u  outputs [n]: x_{T,0} and u_T; [m][n] (one row per worker) when no_average is set.
  *   dbar      optional [T][tau][n]: the worker-mean direction (1/m) sum_i d^{(i)}_{t,k}
  *             (always accumulated in binary64), for the identities of the paper's
  *             "Equivalent Updates" section.
