@@ -105,6 +105,10 @@ typedef struct {
   float x_init;                   /* x_{0,0} in every coordinate                 */
   uint32_t n_tensors;             /* optional segment table: number of parameter tensors */
   const uint64_t *tensor_sizes;   /* HOST array of n_tensors sizes summing to P, or NULL */
+  int32_t no_average;             /* 0: Algorithm 1 as printed. 1: the variant of the paper's Section 6
+                                     that skips the exact average: every worker applies Eq. (2), (3) to
+                                     its own x_{t,tau}; anchor and u are then [m, pitch], one row per
+                                     worker, and SLOWMO_BUF_AVERAGE is refused (EINVAL)                */
 } slowmo_config;
 
 /* Device tensors borrowed from the caller (see "Layout" above). */
@@ -112,8 +116,8 @@ typedef struct {
   float *x;       /* [m, pitch]                                         */
   float *h;       /* [m, pitch]                                         */
   float *v;       /* [m, pitch]; required for Adam, may be NULL else    */
-  float *anchor;  /* [pitch]                                            */
-  float *u;       /* [pitch]                                            */
+  float *anchor;  /* [pitch]; [m, pitch] with no_average                */
+  float *u;       /* [pitch]; [m, pitch] with no_average                */
   float *a;       /* [pitch];    required in generated mode, else NULL  */
   float *c;       /* [m, pitch]; required in generated mode, else NULL  */
   uint64_t pitch; /* row length in elements                             */
@@ -179,6 +183,9 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad);
  *   buffers    reset: h = v = 0 and l = 0; maintain: untouched;
  *              average: h^{(i)} = (sum over i in order) / m for every i, same for v
  * 1/gamma_t and alpha*gamma_t are formed in binary64 on the host and rounded once.
+ * With no_average set there is no average and no broadcast: per worker i,
+ *   u^{(i)} = fma(beta, u^{(i)}, (anchor^{(i)} - x^{(i)}) * (1/gamma_t)) ;
+ *   anchor^{(i)} = fma(-(alpha*gamma_t), u^{(i)}, anchor^{(i)}) ; x^{(i)} = anchor^{(i)}.
  * Advances the outer counter t and sets k = 0.
  */
 int slowmo_outer_step(slowmo_ctx *ctx);

@@ -43,7 +43,7 @@ class Config(C.Structure):
         ("seed", C.c_uint64),
         ("a_lo", C.c_float), ("a_hi", C.c_float), ("c_std", C.c_float), ("sigma", C.c_float),
         ("x_init", C.c_float),
-        ("n_tensors", C.c_uint32), ("tensor_sizes", C.POINTER(C.c_uint64)),
+        ("n_tensors", C.c_uint32), ("tensor_sizes", C.POINTER(C.c_uint64)), ("no_average", C.c_int32),
     ]
 
 
@@ -103,13 +103,14 @@ def _check(status, what):
 
 def make_config(*, P, m, tau, alpha=1.0, beta=0.0, gamma=0.1, base="nesterov", mu=0.0, weight_decay=0.0,
                 adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, buffer_policy="reset", grad_mode="generated",
-                seed=0, a_lo=0.5, a_hi=2.0, c_std=1.0, sigma=0.0, x_init=0.0, tensor_sizes=None, **_ignored):
+                seed=0, a_lo=0.5, a_hi=2.0, c_std=1.0, sigma=0.0, x_init=0.0, tensor_sizes=None, no_average=False,
+                **_ignored):
     """Fill the C config from paper-notation keyword arguments (see include/slowmo.h)."""
     cfg = Config(P, m, tau, alpha, beta, gamma, BASE[base] if isinstance(base, str) else base, mu,
                  weight_decay, adam_b1, adam_b2, adam_eps,
                  POLICY[buffer_policy] if isinstance(buffer_policy, str) else buffer_policy,
                  GRAD[grad_mode] if isinstance(grad_mode, str) else grad_mode, seed, a_lo, a_hi, c_std,
-                 sigma, x_init, 0, None)
+                 sigma, x_init, 0, None, 1 if no_average else 0)
     if tensor_sizes is not None:
         arr = (C.c_uint64 * len(tensor_sizes))(*[int(s) for s in tensor_sizes])
         cfg._keep = arr
@@ -161,8 +162,10 @@ class SlowMo:
         generated = self.cfg.grad_mode == GRAD["generated"]
         self._raw = {}
         self.t = {}
+        self.outer_rows = self.m if self.cfg.no_average else 1
         for name, rows, need in (("x", self.m, True), ("h", self.m, True), ("v", self.m, adam),
-                                 ("anchor", 1, True), ("u", 1, True), ("a", 1, generated),
+                                 ("anchor", self.outer_rows, True), ("u", self.outer_rows, True),
+                                 ("a", 1, generated),
                                  ("c", self.m, generated)):
             self.t[name] = self._alloc(name, rows) if need else None
         ptr = lambda k: self.t[k].data_ptr() if self.t[k] is not None else None
@@ -231,7 +234,8 @@ class SlowMo:
         """Copy columns [offset, offset+count) of tensor `which` to host (numpy) or to `out`
         (a torch CUDA tensor or pinned/pageable numpy array)."""
         count = self.P - offset if count is None else count
-        rows = 1 if (replica >= 0 or which in ("anchor", "u", "a")) else self.m
+        one_row = which == "a" or (which in ("anchor", "u") and not self.cfg.no_average)
+        rows = 1 if (replica >= 0 or one_row) else self.m
         on_device = 0
         if out is None:
             out = np.empty((rows, count), np.float32)

@@ -283,4 +283,52 @@ outer_step_direct_kernel(const OuterArgs A) {
   }
 }
 
+// ---- K2 without the exact average (Section 6 of the paper) -----------------------------------
+
+// Every worker applies Eq. (2) and Eq. (3) to its own model: u, anchor and x are all
+// [m, pitch] and the kernel is a plain elementwise stream, laid out like the local step
+// (one block = one tile of one row). POLICY: 0 reset (h, v zeroed), 1 maintain.
+template <int NBUF, int POLICY, int U>
+__global__ void __launch_bounds__(kThreads)
+outer_step_noaverage_kernel(const OuterArgs A) {
+  const uint32_t row = blockIdx.x % A.m;
+  const uint32_t tile = blockIdx.x / A.m;
+  const uint32_t v0 = tile * (uint32_t)(kThreads * U) + threadIdx.x;
+  const uint64_t roff = (uint64_t)row * A.pitch;
+  float4 x[U], x0[U], u0[U];
+  bool ok[U];
+#pragma unroll
+  for (int q = 0; q < U; ++q) {
+    const uint32_t vi = v0 + q * kThreads;
+    ok[q] = vi < A.nvec;
+    if (ok[q]) {
+      const uint64_t off = roff + 4ull * vi;
+      x[q] = ld_stream(A.x + off);
+      x0[q] = ld_stream(A.anchor + off);
+      u0[q] = ld_stream(A.u + off);
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < U; ++q) {
+    if (!ok[q]) continue;
+    float4 un, xn;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      // Eq. (2), (3) with the worker's own x_{t,tau} in place of the average
+      const float ue = __fmaf_rn(A.beta, comp(u0[q], e), __fmul_rn(__fsub_rn(comp(x0[q], e), comp(x[q], e)), A.inv_gamma));
+      comp(un, e) = ue;
+      comp(xn, e) = __fmaf_rn(A.neg_alpha_gamma, ue, comp(x0[q], e));
+    }
+    const uint64_t off = roff + 4ull * (v0 + q * kThreads);
+    st_stream(A.u + off, un);
+    st_stream(A.anchor + off, xn);
+    st_stream(A.x + off, xn);
+    if (POLICY == 0) {
+      const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+      st_stream(A.h + off, zero);
+      if (NBUF == 2) st_stream(A.v + off, zero);
+    }
+  }
+}
+
 }  // namespace slowmo

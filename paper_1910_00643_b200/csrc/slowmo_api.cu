@@ -104,10 +104,11 @@ int flush_pending(slowmo_ctx *ctx) {
 // Resolve a tensor id to (base pointer, rows); NULL if the tensor does not exist here.
 float *tensor_base(slowmo_ctx *ctx, int which, uint32_t *rows) {
   const slowmo_buffers &b = ctx->buf;
+  const uint32_t outer_rows = ctx->cfg.no_average ? ctx->cfg.m : 1;  // per-worker anchor and u without the average
   switch (which) {
     case SLOWMO_T_X: *rows = ctx->cfg.m; return b.x;
-    case SLOWMO_T_ANCHOR: *rows = 1; return b.anchor;
-    case SLOWMO_T_U: *rows = 1; return b.u;
+    case SLOWMO_T_ANCHOR: *rows = outer_rows; return b.anchor;
+    case SLOWMO_T_U: *rows = outer_rows; return b.u;
     case SLOWMO_T_H: *rows = ctx->cfg.m; return b.h;
     case SLOWMO_T_V: *rows = ctx->cfg.m; return b.v;
     case SLOWMO_T_A: *rows = 1; return b.a;
@@ -155,6 +156,8 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   if (cfg->P == 0 || cfg->m == 0 || cfg->tau == 0) return SLOWMO_EINVAL;
   if (cfg->base < SLOWMO_BASE_NESTEROV || cfg->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
   if (is_sgp(cfg->base) && cfg->m > kSgpMaxWorkers) return SLOWMO_ENOTIMPL;
+  if (cfg->no_average != 0 && cfg->no_average != 1) return SLOWMO_EINVAL;
+  if (cfg->no_average && cfg->buffer_policy == SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
   if (cfg->P > (1ull << 32) - 4096) return SLOWMO_EINVAL;  // columns are indexed with 32 bits
   if (!finite_pos(cfg->alpha) || !unit_interval(cfg->beta) || !finite_pos(cfg->gamma)) return SLOWMO_EINVAL;
   if (cfg->buffer_policy < SLOWMO_BUF_RESET || cfg->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
@@ -237,9 +240,11 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   const size_t row_bytes = (size_t)ctx->nvec * 4 * sizeof(float);
   const size_t pitch_bytes = buf->pitch * sizeof(float);
   fill_value_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->x, buf->pitch, ctx->nvec, cfg->x_init);
-  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, 1), 1), kThreads, 0, ctx->stream>>>(buf->anchor, buf->pitch, ctx->nvec, cfg->x_init);
+  const uint32_t outer_rows = cfg->no_average ? m : 1;
+  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, outer_rows), outer_rows), kThreads, 0, ctx->stream>>>(
+      buf->anchor, buf->pitch, ctx->nvec, cfg->x_init);
   e = cudaGetLastError();
-  if (e == cudaSuccess) e = cudaMemsetAsync(buf->u, 0, row_bytes, ctx->stream);
+  if (e == cudaSuccess) e = cudaMemset2DAsync(buf->u, pitch_bytes, 0, row_bytes, outer_rows, ctx->stream);
   if (e == cudaSuccess) e = cudaMemset2DAsync(buf->h, pitch_bytes, 0, row_bytes, m, ctx->stream);
   if (e == cudaSuccess && buf->v) e = cudaMemset2DAsync(buf->v, pitch_bytes, 0, row_bytes, m, ctx->stream);
   if (e == cudaSuccess && generated) {
@@ -309,7 +314,7 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     ctx->k += 1;
     // fused variant: step tau-1 is taken inside the outer-step kernel
     if (ctx->outer_variant == SLOWMO_OUTER_FUSED && ctx->k == c.tau && (!generated || c.m <= kInlineKeys) &&
-        !is_sgp(c.base)) {
+        !is_sgp(c.base) && !c.no_average) {
       ctx->pending = A;
       ctx->pending_last = true;
       break;
@@ -347,7 +352,18 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
   if (ctx->pending_last && variant != SLOWMO_OUTER_FUSED) {
     if (int rc = flush_pending(ctx)) return rc;
   }
-  if (ctx->pending_last) {
+  if (c.no_average) {
+    const uint32_t per_tile = kThreads * kLocalUnroll;
+    const uint32_t blocks = ((ctx->nvec + per_tile - 1) / per_tile) * c.m;
+    const bool reset = c.buffer_policy == SLOWMO_BUF_RESET;
+    if (nbuf == 1) {
+      if (reset) outer_step_noaverage_kernel<1, 0, kLocalUnroll><<<blocks, kThreads, 0, ctx->stream>>>(A);
+      else outer_step_noaverage_kernel<1, 1, kLocalUnroll><<<blocks, kThreads, 0, ctx->stream>>>(A);
+    } else {
+      if (reset) outer_step_noaverage_kernel<2, 0, kLocalUnroll><<<blocks, kThreads, 0, ctx->stream>>>(A);
+      else outer_step_noaverage_kernel<2, 1, kLocalUnroll><<<blocks, kThreads, 0, ctx->stream>>>(A);
+    }
+  } else if (ctx->pending_last) {
     ctx->pending_last = false;
     launch_last_step_outer(ctx->pending, A, c.base == SLOWMO_BASE_ADAM, c.grad_mode == SLOWMO_GRAD_GENERATED,
                            c.buffer_policy, ctx->stream);

@@ -32,7 +32,7 @@ def _gather(s, key, j):
     import torch
     idx = torch.as_tensor(np.asarray(j, dtype=np.int64), device="cuda")
     t = s.t[key]
-    two_d = key in ("x", "h", "v", "c")
+    two_d = key in ("x", "h", "v", "c") or (key in ("anchor", "u") and s.cfg.no_average)
     out = t.view(s.m if two_d else 1, s.pitch).index_select(1, idx).cpu().numpy()
     return out if two_d else out[0]
 
@@ -326,6 +326,47 @@ def test_full_size_sgp_workloads_on_sampled_coordinates(name):
     _check_against_oracle(s, w, j, exact=True)
     x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
     assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    s.close()
+    del s
+    torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------- variant without the exact average (Section 6)
+
+@pytest.mark.parametrize("base,policy", [("nesterov", "reset"), ("nesterov", "maintain"), ("adam", "maintain"),
+                                         ("adam", "reset"), ("sgp_nesterov", "reset"), ("sgp_adam", "maintain")])
+@pytest.mark.parametrize("m", [1, 3, 8])
+def test_no_average_small_runs_match_oracle(base, policy, m):
+    w = workloads.workload("tiny", P=2 * 1024 + 37, m=m, tau=4, T=3, base=base, buffer_policy=policy, alpha=0.9,
+                           beta=0.6, gamma=0.01 if "adam" in base else 0.05, weight_decay=1e-3, adam_b1=0.9,
+                           adam_b2=0.98, adam_eps=1e-8, seed=12, no_average=True)
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", "fused")      # has no effect without the average
+    s.run(w["T"])
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.get_params("anchor").shape == (m, w["P"]) and s.get_params("u", replica=m - 1).shape == (1, w["P"])
+    assert s.guards_intact()
+    s.close()
+
+
+def test_no_average_refuses_the_average_policy():
+    from paper_1910_00643_b200 import SlowMoError, binding
+    with pytest.raises(SlowMoError) as e:
+        _slowmo(workloads.workload("tiny", buffer_policy="average", no_average=True))
+    assert e.value.status == binding.EINVAL
+
+
+def test_full_size_sgp_without_the_average_on_sampled_coordinates():
+    import torch
+    w = workloads.workload("sgp_resnet50", T=2, no_average=True)
+    s = _slowmo(w)
+    s.run(w["T"])
+    j = workloads.sample_coordinates(w["P"], 1 << 12, seed=4)
+    _check_against_oracle(s, w, j, exact=True)
+    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
+    anchor = s.t["anchor"].view(w["m"], s.pitch)[:, :w["P"]]
+    assert torch.equal(x, anchor)                       # each worker restarts from its own outer iterate
+    assert not bool((x == x[0:1]).all())                # and the workers no longer agree
     s.close()
     del s
     torch.cuda.empty_cache()
