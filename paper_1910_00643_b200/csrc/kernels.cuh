@@ -22,6 +22,12 @@ constexpr int kThreads = 256;
 #ifndef SLOWMO_LOCAL_MIN_BLOCKS
 #define SLOWMO_LOCAL_MIN_BLOCKS 1  // __launch_bounds__ minimum resident blocks per SM
 #endif
+#ifndef SLOWMO_LOCAL_LAYOUT
+#define SLOWMO_LOCAL_LAYOUT 0   // 0: choose by m; 1: always row tiles; 2: column owner whenever possible
+#endif
+#ifndef SLOWMO_LOCAL_COL_ROWS
+#define SLOWMO_LOCAL_COL_ROWS 4  // rows in flight per thread in the column-owner layout (Nesterov; Adam half)
+#endif
 #ifndef SLOWMO_STREAM_HINT
 #define SLOWMO_STREAM_HINT 0    // 1: evict-first (.cs) loads and stores, 0: default policy
 #endif
@@ -198,6 +204,57 @@ local_step_kernel(const LocalArgs A) {
     st_stream(A.x + off, x[u]);
     st_stream(A.h + off, h[u]);
     if (BASE == 1) st_stream(A.v + off, v[u]);
+  }
+}
+
+// Column-owner layout of the same step: one thread owns a 4-column group and walks all m rows,
+// ROWS at a time. The curvature is loaded once per column (instead of once per row from L2)
+// and consecutive rows of a thread's loads are independent, so fewer threads keep as many
+// bytes in flight. Same arithmetic per element as local_step_kernel: results are identical.
+// Needs the row keys in the kernel arguments (m <= kInlineKeys) in generated mode.
+template <int BASE, int GRAD, int ROWS>
+__global__ void __launch_bounds__(kThreads)
+local_step_cols_kernel(const LocalArgs A) {
+  const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
+  if (vi >= A.nvec) return;
+  const uint64_t col = 4ull * vi;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (GRAD == 0) a = ld_shared_row(A.a + col);
+  for (uint32_t i0 = 0; i0 < A.m; i0 += ROWS) {
+    float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) {
+      if (i0 + q < A.m) {
+        const uint64_t off = (uint64_t)(i0 + q) * A.pitch + col;
+        x[q] = ld_stream(A.x + off);
+        h[q] = ld_stream(A.h + off);
+        if (BASE == 1) v[q] = ld_stream(A.v + off);
+        s[q] = ld_stream(A.src + off);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < ROWS; ++q) {
+      const uint32_t i = i0 + q;
+      if (i >= A.m) break;
+      float4 g;
+      if (GRAD == 0) {
+        const uint64_t st = A.keys[i] + kGoldenGamma * (2ull * vi + 1);
+        float4 z;
+        word_to_normal_pair(mix64(st), z.x, z.y);
+        word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(A.sigma, comp(z, e)));
+      } else {
+        g = s[q];
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) base_step<BASE>(A, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
+      const uint64_t off = (uint64_t)i * A.pitch + col;
+      st_stream(A.x + off, x[q]);
+      st_stream(A.h + off, h[q]);
+      if (BASE == 1) st_stream(A.v + off, v[q]);
+    }
   }
 }
 
