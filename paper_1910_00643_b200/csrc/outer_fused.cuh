@@ -10,6 +10,13 @@
 #pragma once
 #include "kernels.cuh"
 
+#ifndef SLOWMO_FUSED_ROWS
+#define SLOWMO_FUSED_ROWS 2        // rows in flight per thread (Nesterov; Adam uses half)
+#endif
+#ifndef SLOWMO_FUSED_MIN_BLOCKS
+#define SLOWMO_FUSED_MIN_BLOCKS 4  // __launch_bounds__ minimum resident blocks per SM
+#endif
+
 namespace slowmo {
 
 __device__ __forceinline__ void add_in_order(float4 &s, const float4 &v, bool first) {
@@ -30,7 +37,7 @@ __device__ __forceinline__ float4 div4(const float4 &s, float d) {
 // One thread = one 4-element column group, all m rows. ROWS rows are loaded together.
 // Requires m <= kInlineKeys in generated mode (the launcher falls back otherwise).
 template <int BASE, int GRAD, int POLICY, int ROWS>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, SLOWMO_FUSED_MIN_BLOCKS)
 last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
   if (vi >= O.nvec) return;
@@ -110,7 +117,7 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
 template <int BASE, int GRAD>
 inline void launch_last_step_outer_policy(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
   const uint32_t blocks = (O.nvec + kThreads - 1) / kThreads;
-  constexpr int ROWS = BASE == 1 ? 2 : 4;
+  constexpr int ROWS = BASE == 1 ? SLOWMO_FUSED_ROWS / 2 : SLOWMO_FUSED_ROWS;
   switch (policy) {
     case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
     case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
