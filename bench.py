@@ -30,8 +30,9 @@ FALLBACK_HBM_GBS = 6650.0
 # algorithmic bytes, from ncu captures of small cases of the current kernels (profiles/);
 # traffic grows in proportion to m*P, so the ratio carries to the full launch. None = no capture
 # of the kernel as it stands.
-NCU_TRAFFIC_RATIO = {("local_step", "generated"): 0.962, ("local_step", "supplied"): 0.980,
-                     ("outer_step", "average"): 0.951, ("outer_step", "reset"): 0.973}
+NCU_TRAFFIC_RATIO = {("local_step", "generated"): 0.961, ("local_step", "supplied"): 0.980,
+                     ("outer_step", "average"): 0.952, ("outer_step", "reset"): 0.973,
+                     ("last_step_outer", "generated-average"): 0.975, ("last_step_outer", "supplied-reset"): 0.983}
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -276,7 +277,7 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
         total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant == "fused")
         if variant == "fused":
             out["last_step_outer_fused"] = roofline("last_step_outer", fused_outer_step_bytes(w), outer, peak,
-                                                    peak_kind)
+                                                    peak_kind, "supplied-reset")
         else:
             out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind, "supplied")
             out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind,
@@ -368,7 +369,8 @@ def run_ours(args):
         "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
                              w["grad_mode"] if w["base"] == "nesterov" else None),
         "roofline_outer_step": (
-            roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind) if fused else
+            roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind,
+                     f"{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if fused else
             roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
                      w["buffer_policy"] if args.outer_variant == "direct" and w["base"] == "nesterov"
                      and w["buffer_policy"] != "maintain" else None)),
