@@ -286,6 +286,22 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
     s.close()
     del s
     torch.cuda.empty_cache()
+    # the workload is defined as a sweep over tau: whole-run updates/s at tau = 1 and 48 too (T = 3)
+    sweep = {str(tau): {v: out["updates_per_s_tau%d_%s" % (tau, v)] for v in ("direct", "fused")}}
+    for t_in in (1, 48):
+        wt = workloads.workload("stress_tau12", tau=t_in)
+        s = SlowMo(wt)
+        s.alloc_gradient()
+        s.fill_gradient()
+        sweep[str(t_in)] = {}
+        for variant in ("direct", "fused"):
+            s.set_variant("outer", variant)
+            total, _, _ = time_steps(s, wt, wt["T"], 1, s.grad, fused=variant == "fused")
+            sweep[str(t_in)][variant] = wt["m"] * wt["P"] * t_in * wt["T"] / (total * 1e-3)
+        s.close()
+        del s
+        torch.cuda.empty_cache()
+    out["updates_per_s_by_tau"] = sweep
     return out
 
 

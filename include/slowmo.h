@@ -279,6 +279,14 @@ int slowmo_outer_step_static(float *x, float *h, float *v, float *anchor, float 
                              uint64_t P, uint32_t m, int32_t base, int32_t buffer_policy, float alpha,
                              float beta, float gamma_t, void *cuda_stream, int wait);
 
+/*
+ * Test hook for the error path of the bounded device-side waits: enqueues a one-block kernel
+ * that waits, with the pipeline's own try loop limited to `tries` (1 .. 2^20) attempts, on a
+ * barrier that nothing completes, and records the timeout. The next slowmo_sync_status
+ * returns SLOWMO_ETIMEOUT once and clears the record; the context and the GPU stay usable.
+ */
+int slowmo_debug_wait_timeout(slowmo_ctx *ctx, uint32_t tries);
+
 const char *slowmo_strerror(int status);
 int slowmo_last_cuda_error(slowmo_ctx *ctx);
 

@@ -24,7 +24,7 @@ EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_oute
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
-           "slowmo_outer_step_static"]
+           "slowmo_outer_step_static", "slowmo_debug_wait_timeout"]
 
 
 class SlowMoError(RuntimeError):
@@ -79,6 +79,7 @@ def lib():
             "slowmo_set_variant": [vp, C.c_int, C.c_int],
             "slowmo_sync_status": [vp],
             "slowmo_last_cuda_error": [vp],
+            "slowmo_debug_wait_timeout": [vp, u32],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -224,6 +225,9 @@ class SlowMo:
 
     def sync_status(self):
         _check(lib().slowmo_sync_status(self.ctx), "slowmo_sync_status")
+
+    def debug_wait_timeout(self, tries=4096):
+        _check(lib().slowmo_debug_wait_timeout(self.ctx, tries), "slowmo_debug_wait_timeout")
 
     def counters(self):
         t, k, l = C.c_uint64(), C.c_uint32(), C.c_uint64()

@@ -291,6 +291,20 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
   __syncthreads();
 }
 
+// Test hook for the bounded-wait path: one CTA waits on an mbarrier that nothing ever
+// completes, with the same try loop as the pipeline (bound given by the caller), records the
+// timeout in the status block and returns. The context stays usable.
+__global__ void bounded_wait_probe_kernel(int *status, uint32_t tries) {
+  __shared__ unsigned long long bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    bool done = false;
+    for (uint32_t i = 0; i < tries && !done; ++i) done = mbar_try_wait(&bar, 0);
+    if (!done && atomicExch(status, 1) == 0) status[1] = 99;
+  }
+}
+
 inline cudaError_t outer_staged_configure() {
   const int bytes = (int)sizeof(StagedSmem);
   cudaError_t e = cudaSuccess;

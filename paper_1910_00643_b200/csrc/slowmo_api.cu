@@ -487,6 +487,13 @@ int slowmo_sync_status(slowmo_ctx *ctx) {
   return SLOWMO_OK;
 }
 
+int slowmo_debug_wait_timeout(slowmo_ctx *ctx, uint32_t tries) {
+  if (!ctx || tries == 0 || tries > (1u << 20)) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  bounded_wait_probe_kernel<<<1, 32, 0, ctx->stream>>>(ctx->status_dev, tries);
+  return check_launch(ctx);
+}
+
 const char *slowmo_strerror(int status) {
   switch (status) {
     case SLOWMO_OK: return "ok";

@@ -417,6 +417,23 @@ def test_call_order_and_argument_errors():
     s.close()
 
 
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
+    from paper_1910_00643_b200 import SlowMoError, binding
+    w = workloads.workload("tiny", P=3000)
+    s = _slowmo(w)
+    s.set_variant("outer", "staged")
+    s.run(1)
+    s.sync_status()                       # clean so far
+    s.debug_wait_timeout(4096)            # a wait on a barrier nothing completes
+    with pytest.raises(SlowMoError) as e:
+        s.sync_status()
+    assert e.value.status == binding.ETIMEOUT
+    s.sync_status()                       # the record is cleared, the context still works
+    s.run(2)
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    s.close()
+
+
 def test_get_and_set_params_round_trip():
     import torch
     w = workloads.workload("tiny", P=3001, m=3)

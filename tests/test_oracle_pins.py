@@ -388,3 +388,16 @@ def test_coordinate_lists_and_ranges_agree():
     some = oracle.run(cfg, j=pick)
     assert np.array_equal(some["x"], full["x"][:, pick.astype(int)])
     assert np.array_equal(some["u"], full["u"][pick.astype(int)])
+
+
+def test_binary32_oracle_matches_its_frozen_outputs():
+    # regression net: the stored bit patterns were written by tests/golden/make_oracle_golden.py from
+    # the oracle itself; a mismatch means the oracle's arithmetic changed
+    import importlib.util
+    import os
+    here = os.path.join(os.path.dirname(__file__), "golden")
+    spec = importlib.util.spec_from_file_location("make_oracle_golden", os.path.join(here, "make_oracle_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    stored = [l.strip() for l in open(os.path.join(here, "oracle_f32_cases.txt")) if not l.startswith("#")]
+    assert stored == list(mod.lines())
