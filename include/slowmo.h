@@ -190,6 +190,21 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad);
  */
 int slowmo_outer_step(slowmo_ctx *ctx);
 
+/*
+ * One whole outer iteration of Algorithm 1 (tau local steps, then the outer step) with HOST
+ * input and output, pipelined over column windows: the per-worker problem data c [m, P]
+ * (dense, no padding; pinned memory for the copies to overlap) is uploaded window by window on
+ * a copy stream while the windows already on the device run their tau + 1 kernels on the
+ * context's stream, and each window's new outer iterate is written to anchor_host ([P], or
+ * [m, P] with no_average) on a second copy stream. Every statement of Algorithm 1 is elementwise
+ * in the coordinate, so the windows are independent and the result is bit-identical to
+ * slowmo_set_params(c) + slowmo_local_steps(tau) + slowmo_outer_step + slowmo_get_params(anchor).
+ * `chunks` (1..1024) is the number of windows asked for; windows are whole 2048-column tiles.
+ * Generated-gradient mode only (ENOTIMPL otherwise); legal only at k = 0 (ESTATE). Waits for
+ * completion before returning.
+ */
+int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks);
+
 /* Change the base learning rate (a schedule's gamma_t). Legal only between outer
  * iterations, i.e. when k = 0 (ESTATE otherwise). EINVAL unless gamma > 0 and finite. */
 int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t);

@@ -24,7 +24,7 @@ EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_oute
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
-           "slowmo_outer_step_static", "slowmo_debug_wait_timeout"]
+           "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host"]
 
 
 class SlowMoError(RuntimeError):
@@ -80,6 +80,7 @@ def lib():
             "slowmo_sync_status": [vp],
             "slowmo_last_cuda_error": [vp],
             "slowmo_debug_wait_timeout": [vp, u32],
+            "slowmo_iteration_host": [vp, vp, vp, u32],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -216,6 +217,12 @@ class SlowMo:
 
     def outer_step(self):
         _check(lib().slowmo_outer_step(self.ctx), "slowmo_outer_step")
+
+    def iteration_host(self, c_host, anchor_host, chunks=8):
+        """slowmo_iteration_host: one outer iteration with host input c [m, P] and host output
+        anchor (torch CPU tensors, pinned for overlap, or numpy arrays)."""
+        ptr = lambda a: a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
+        _check(lib().slowmo_iteration_host(self.ctx, ptr(c_host), ptr(anchor_host), chunks), "slowmo_iteration_host")
 
     def set_gamma(self, gamma):
         _check(lib().slowmo_set_gamma(self.ctx, gamma), "slowmo_set_gamma")

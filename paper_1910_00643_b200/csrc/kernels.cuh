@@ -116,7 +116,8 @@ struct LocalArgs {
   const float *src;       // generated mode: centres c [m, pitch]; supplied mode: gradient G [m, pitch]
   const float *a;         // [pitch], generated mode
   uint64_t pitch;
-  uint32_t nvec;          // 4-element column groups per row
+  uint32_t nvec;          // 4-element column groups per row (of the column window being processed)
+  uint32_t vec0;          // index of the window's first column group in the whole vector (noise index)
   uint32_t m;
   uint64_t seed, t;       // outer iteration, for the noise key
   uint32_t k;             // inner step, for the noise key
@@ -188,7 +189,7 @@ local_step_kernel(const LocalArgs A) {
     float4 g;
     if (GRAD == 0) {
       // columns 4vi..4vi+3 take the Box-Muller pairs of words 2vi and 2vi+1 of the row's stream
-      const uint64_t st = key + kGoldenGamma * (2ull * vi + 1);
+      const uint64_t st = key + kGoldenGamma * (2ull * (A.vec0 + vi) + 1);
       float4 z;
       word_to_normal_pair(mix64(st), z.x, z.y);
       word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
@@ -238,7 +239,7 @@ local_step_cols_kernel(const LocalArgs A) {
       if (i >= A.m) break;
       float4 g;
       if (GRAD == 0) {
-        const uint64_t st = A.keys[i] + kGoldenGamma * (2ull * vi + 1);
+        const uint64_t st = A.keys[i] + kGoldenGamma * (2ull * (A.vec0 + vi) + 1);
         float4 z;
         word_to_normal_pair(mix64(st), z.x, z.y);
         word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);

@@ -57,7 +57,7 @@ sgp_step_kernel(const LocalArgs L, uint32_t hops) {
       if (i >= m) break;
       float4 g;
       if (GRAD == 0) {
-        const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * vi + 1);
+        const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * (L.vec0 + vi) + 1);
         float4 z;
         word_to_normal_pair(mix64(st), z.x, z.y);
         word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);

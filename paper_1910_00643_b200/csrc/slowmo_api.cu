@@ -23,6 +23,8 @@ struct slowmo_ctx {
   slowmo_buffers buf;
   cudaStream_t stream;
   uint32_t nvec;             // 4-element column groups per row: ceil(P/4)
+  uint32_t win_vec0, win_nvec;  // column window that launches cover (whole vector except inside slowmo_iteration_host)
+  cudaStream_t copy_in, copy_out;  // created on first use by slowmo_iteration_host
   uint64_t t;                // outer iteration
   uint32_t k;                // inner steps taken in this outer iteration
   uint64_t l;                // Adam steps since the buffers were last zero
@@ -77,18 +79,18 @@ template <int BASE, int GRAD>
 void launch_local(slowmo_ctx *ctx, const LocalArgs &A) {
   if (use_column_owner(ctx)) {
     constexpr int ROWS = BASE == 1 ? SLOWMO_LOCAL_COL_ROWS / 2 : SLOWMO_LOCAL_COL_ROWS;
-    const uint32_t blocks = (ctx->nvec + kThreads - 1) / kThreads;
+    const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
     local_step_cols_kernel<BASE, GRAD, ROWS><<<blocks, kThreads, 0, ctx->stream>>>(A);
     return;
   }
   const uint32_t per_tile = kThreads * kLocalUnroll;
-  const uint32_t tiles = (ctx->nvec + per_tile - 1) / per_tile;
+  const uint32_t tiles = (A.nvec + per_tile - 1) / per_tile;
   local_step_kernel<BASE, GRAD, kLocalUnroll><<<tiles * ctx->cfg.m, kThreads, 0, ctx->stream>>>(A);
 }
 
 template <int NBUF>
 void launch_outer_direct(slowmo_ctx *ctx, const OuterArgs &A) {
-  const uint32_t blocks = (ctx->nvec + kThreads - 1) / kThreads;
+  const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
   switch (ctx->cfg.buffer_policy) {
     case SLOWMO_BUF_RESET: outer_step_direct_kernel<NBUF, 0><<<blocks, kThreads, 0, ctx->stream>>>(A); break;
     case SLOWMO_BUF_MAINTAIN: outer_step_direct_kernel<NBUF, 1><<<blocks, kThreads, 0, ctx->stream>>>(A); break;
@@ -206,6 +208,9 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   ctx->buf = *buf;
   ctx->stream = (cudaStream_t)cuda_stream;
   ctx->nvec = (uint32_t)nvec;
+  ctx->win_vec0 = 0;
+  ctx->win_nvec = (uint32_t)nvec;
+  ctx->copy_in = ctx->copy_out = nullptr;
   ctx->t = 0;
   ctx->k = 0;
   ctx->l = 0;
@@ -282,6 +287,8 @@ int slowmo_destroy(slowmo_ctx *ctx) {
   if (!ctx) return SLOWMO_EINVAL;
   flush_pending(ctx);
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->copy_in) cudaStreamDestroy(ctx->copy_in);
+  if (ctx->copy_out) cudaStreamDestroy(ctx->copy_out);
   if (ctx->status_dev) cudaFree(ctx->status_dev);
   delete ctx;
   return SLOWMO_OK;
@@ -296,14 +303,16 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
   if (grad && !aligned16(grad)) return SLOWMO_EALIGN;
   if ((uint64_t)ctx->k + n > c.tau) return SLOWMO_ESTATE;
 
+  const uint64_t woff = 4ull * ctx->win_vec0;  // first column of the window
   LocalArgs A;
-  A.x = ctx->buf.x;
-  A.h = ctx->buf.h;
-  A.v = ctx->buf.v;
-  A.src = generated ? ctx->buf.c : grad;
-  A.a = ctx->buf.a;
+  A.x = ctx->buf.x + woff;
+  A.h = ctx->buf.h + woff;
+  A.v = ctx->buf.v ? ctx->buf.v + woff : nullptr;
+  A.src = (generated ? ctx->buf.c : grad) + woff;
+  A.a = ctx->buf.a ? ctx->buf.a + woff : nullptr;
   A.pitch = ctx->buf.pitch;
-  A.nvec = ctx->nvec;
+  A.nvec = ctx->win_nvec;
+  A.vec0 = ctx->win_vec0;
   A.m = c.m;
   A.seed = c.seed;
   A.neg_gamma = -ctx->gamma;
@@ -348,14 +357,15 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
   const slowmo_config &c = ctx->cfg;
   if (ctx->k != c.tau) return SLOWMO_ESTATE;
 
+  const uint64_t woff = 4ull * ctx->win_vec0;
   OuterArgs A;
-  A.x = ctx->buf.x;
-  A.h = ctx->buf.h;
-  A.v = ctx->buf.v;
-  A.anchor = ctx->buf.anchor;
-  A.u = ctx->buf.u;
+  A.x = ctx->buf.x + woff;
+  A.h = ctx->buf.h + woff;
+  A.v = ctx->buf.v ? ctx->buf.v + woff : nullptr;
+  A.anchor = ctx->buf.anchor + woff;
+  A.u = ctx->buf.u + woff;
   A.pitch = ctx->buf.pitch;
-  A.nvec = ctx->nvec;
+  A.nvec = ctx->win_nvec;
   A.m = c.m;
   A.beta = c.beta;
   A.inv_gamma = (float)(1.0 / (double)ctx->gamma);
@@ -370,7 +380,7 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
   }
   if (c.no_average) {
     const uint32_t per_tile = kThreads * kLocalUnroll;
-    const uint32_t blocks = ((ctx->nvec + per_tile - 1) / per_tile) * c.m;
+    const uint32_t blocks = ((A.nvec + per_tile - 1) / per_tile) * c.m;
     const bool reset = c.buffer_policy == SLOWMO_BUF_RESET;
     if (nbuf == 1) {
       if (reset) outer_step_noaverage_kernel<1, 0, kLocalUnroll><<<blocks, kThreads, 0, ctx->stream>>>(A);
@@ -398,6 +408,69 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
     ctx->pow_b1 = ctx->pow_b2 = 1.0;
   }
   return SLOWMO_OK;
+}
+
+int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks) {
+  if (!ctx || !c_host || !anchor_host || chunks == 0 || chunks > 1024) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  const slowmo_config &c = ctx->cfg;
+  if (c.grad_mode != SLOWMO_GRAD_GENERATED) return SLOWMO_ENOTIMPL;
+  if (ctx->k != 0 || ctx->pending_last) return SLOWMO_ESTATE;
+  cudaError_t e = cudaSuccess;
+  if (!ctx->copy_in) e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
+  if (e == cudaSuccess && !ctx->copy_out) e = cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking);
+  if (e != cudaSuccess) return cuda_fail(ctx, e);
+
+  // windows of whole 2048-column tiles so that every window start keeps the 16-byte (and tile) alignment
+  uint32_t win = (ctx->nvec + chunks - 1) / chunks;
+  win = (win + 511u) / 512u * 512u;
+  const uint32_t nwin = (ctx->nvec + win - 1) / win;
+  const uint32_t outer_rows = c.no_average ? c.m : 1;
+  const size_t dpitch = ctx->buf.pitch * sizeof(float), hpitch = (size_t)c.P * sizeof(float);
+  std::vector<cudaEvent_t> ev(2 * (size_t)nwin + 1, nullptr);
+  for (auto &x : ev)
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&x, cudaEventDisableTiming);
+  int rc = SLOWMO_OK;
+  // uploads must not overtake earlier work of this context that still reads the centres
+  if (e == cudaSuccess) e = cudaEventRecord(ev[2 * nwin], ctx->stream);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_in, ev[2 * nwin], 0);
+
+  const uint64_t t0 = ctx->t, l0 = ctx->l;
+  const double p1 = ctx->pow_b1, p2 = ctx->pow_b2;
+  for (uint32_t w = 0; w < nwin && e == cudaSuccess && rc == SLOWMO_OK; ++w) {
+    const uint32_t vec0 = w * win, nv = ctx->nvec - vec0 < win ? ctx->nvec - vec0 : win;
+    const uint64_t col0 = 4ull * vec0;
+    const uint64_t cols = c.P - col0 < 4ull * nv ? c.P - col0 : 4ull * nv;  // host arrays have no padding
+    e = cudaMemcpy2DAsync(ctx->buf.c + col0, dpitch, c_host + col0, hpitch, cols * sizeof(float), c.m,
+                          cudaMemcpyHostToDevice, ctx->copy_in);
+    if (e == cudaSuccess) e = cudaEventRecord(ev[2 * w], ctx->copy_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, ev[2 * w], 0);
+    if (e != cudaSuccess) break;
+    // the whole outer iteration on this window; every window sees the same counters
+    ctx->t = t0;
+    ctx->k = 0;
+    ctx->l = l0;
+    ctx->pow_b1 = p1;
+    ctx->pow_b2 = p2;
+    ctx->win_vec0 = vec0;
+    ctx->win_nvec = nv;
+    rc = slowmo_local_steps(ctx, c.tau, nullptr);
+    if (rc == SLOWMO_OK) rc = slowmo_outer_step(ctx);
+    if (rc != SLOWMO_OK) break;
+    e = cudaEventRecord(ev[2 * w + 1], ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_out, ev[2 * w + 1], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpy2DAsync(anchor_host + col0, hpitch, ctx->buf.anchor + col0, dpitch, cols * sizeof(float), outer_rows,
+                            cudaMemcpyDeviceToHost, ctx->copy_out);
+  }
+  ctx->win_vec0 = 0;
+  ctx->win_nvec = ctx->nvec;
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->copy_out);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+  for (auto x : ev)
+    if (x) cudaEventDestroy(x);
+  if (rc != SLOWMO_OK) return rc;
+  return cuda_fail(ctx, e);
 }
 
 int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t) {

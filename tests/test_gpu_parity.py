@@ -434,6 +434,40 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     s.close()
 
 
+@pytest.mark.parametrize("name,over,variant,chunks", [
+    ("tiny", dict(P=10_007, m=3, tau=3, buffer_policy="average"), "fused", 3),
+    ("tiny", dict(P=10_007, m=3, tau=3, buffer_policy="reset"), "staged", 4),
+    ("transformer_adam", dict(P=9_001, m=4, tau=2), "direct", 2),
+    ("sgp_resnet50", dict(P=12_345, m=5, tau=4), "direct", 5),
+    ("tiny", dict(P=7_000, m=3, tau=2, buffer_policy="maintain", no_average=True), "direct", 3),
+    ("tiny", dict(P=100, m=2, tau=1), "fused", 8),
+])
+def test_pipelined_host_iteration_equals_the_plain_call_sequence(name, over, variant, chunks):
+    import torch
+    w = workloads.workload(name, **over)
+    P, m = w["P"], w["m"]
+    rng = np.random.Generator(np.random.PCG64(5))
+    a, b = _slowmo(w, guard=64), _slowmo(w, guard=64)
+    for s in (a, b):
+        s.set_variant("outer", variant)
+    rows = m if w.get("no_average") else 1
+    for it in range(3):
+        c_host = torch.from_numpy(rng.standard_normal((m, P)).astype(np.float32)).pin_memory()
+        out_host = torch.empty((rows, P), dtype=torch.float32).pin_memory()
+        a.iteration_host(c_host, out_host, chunks)          # pipelined
+        b.set_params("c", c_host)                            # plain sequence
+        b.local_steps(w["tau"])
+        b.outer_step()
+        ref = b.get_params("anchor")
+        assert np.array_equal(out_host.numpy().view(np.uint32), ref.view(np.uint32)), it
+    for key in _state_keys(w):
+        assert np.array_equal(a.get_params(key).view(np.uint32), b.get_params(key).view(np.uint32)), key
+    assert a.counters() == b.counters()
+    assert a.guards_intact() and b.guards_intact()
+    a.close()
+    b.close()
+
+
 def test_get_and_set_params_round_trip():
     import torch
     w = workloads.workload("tiny", P=3001, m=3)
