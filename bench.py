@@ -75,6 +75,38 @@ def fused_outer_step_bytes(w):
     return per_param * P
 
 
+def lazy_outer_step_bytes(w):
+    """Algorithmic bytes of the fused outer step in the lazy variant: as fused_outer_step_bytes
+    without the m broadcast rows of x and without the reset / averaged buffer rows (the mean goes
+    to one row)."""
+    m, P = w["m"], w["P"]
+    nb = 2 if "adam" in w["base"] else 1
+    per_param = m * (4 + 4 * nb + 4) + 8 + 8
+    if w["grad_mode"] == "generated":
+        per_param += 4
+    if w["buffer_policy"] == "maintain":
+        per_param += 4 * m * nb
+    elif w["buffer_policy"] == "average":
+        per_param += 4 * nb
+    return per_param * P
+
+
+def virtual_first_step_bytes(w):
+    """Algorithmic bytes of the first local step after a lazy outer step: c-or-G of the m rows
+    and the anchor read (plus the buffer rows under "maintain", or the one row of means under
+    "average"), x and the buffers of the m rows written."""
+    m, P = w["m"], w["P"]
+    nb = 2 if "adam" in w["base"] else 1
+    per_param = 4 * m + 4 + 4 * m + 4 * m * nb
+    if w["grad_mode"] == "generated":
+        per_param += 4
+    if w["buffer_policy"] == "maintain":
+        per_param += 4 * m * nb
+    elif w["buffer_policy"] == "average":
+        per_param += 4 * nb
+    return per_param * P
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -174,31 +206,42 @@ def aggregate_throughput(units_this_rank, ms_this_rank, device=None):
 
 # --------------------------------------------------------------------------------- timed loops
 
-def time_steps(s, w, steps, warmup, grad=None, fused=False):
+def time_steps(s, w, steps, warmup, grad=None, fused=False, lazy=False):
     """Device-timed outer iterations. Returns total ms and the per-kernel mean launch ms.
     With the fused variant the last inner step runs inside the outer-step kernel, so an
-    iteration has tau-1 local-step launches."""
+    iteration has tau-1 local-step launches. With the lazy variant the first launch of an
+    iteration (which reads the anchor instead of the rows) is timed apart and returned in
+    time_steps.first_ms; the run ends with slowmo_materialize inside the timed region."""
     import torch
-    local_launches = max(1, w["tau"] - 1) if fused else w["tau"]
+    tau = w["tau"]
+    split_first = lazy and tau >= 3
+    local_launches = (max(1, tau - 1) if fused else tau) - (1 if split_first else 0)
     for _ in range(warmup):
-        s.local_steps(w["tau"], grad)
+        s.local_steps(tau, grad)
         s.outer_step()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    end = torch.cuda.Event(enable_timing=True)
     s.synchronize()
     barrier()
     torch.cuda.synchronize()
     for i in range(steps):
         ev[i][0].record(s.stream)
-        s.local_steps(w["tau"], grad)
+        if split_first:
+            s.local_steps(1, grad)
         ev[i][1].record(s.stream)
-        s.outer_step()
+        s.local_steps(tau - 1 if split_first else tau, grad)
         ev[i][2].record(s.stream)
+        s.outer_step()
+        ev[i][3].record(s.stream)
+    s.materialize()
+    end.record(s.stream)
     s.synchronize()
     torch.cuda.synchronize()
     barrier()
-    total = ev[0][0].elapsed_time(ev[-1][2])
-    local = sum(e[0].elapsed_time(e[1]) for e in ev) / (steps * local_launches)
-    outer = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+    total = ev[0][0].elapsed_time(end)
+    time_steps.first_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / steps if split_first else None
+    local = sum(e[1].elapsed_time(e[2]) for e in ev) / (steps * local_launches)
+    outer = sum(e[2].elapsed_time(e[3]) for e in ev) / steps
     s.sync_status()
     return total, local, outer
 
@@ -271,10 +314,15 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
     s = SlowMo(w)
     s.alloc_gradient()
     s.fill_gradient()
-    for variant in ("direct", "staged", "fused"):
+    for variant in ("direct", "staged", "fused", "lazy"):
         s.set_variant("outer", variant)
-        total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant == "fused")
-        if variant == "fused":
+        total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant in ("fused", "lazy"),
+                                         lazy=variant == "lazy")
+        if variant == "lazy":
+            out["last_step_outer_lazy"] = roofline("last_step_outer", lazy_outer_step_bytes(w), outer, peak, peak_kind)
+            out["first_local_step_lazy"] = roofline("local_step", virtual_first_step_bytes(w), time_steps.first_ms,
+                                                    peak, peak_kind)
+        elif variant == "fused":
             out["last_step_outer_fused"] = roofline("last_step_outer", fused_outer_step_bytes(w), outer, peak,
                                                     peak_kind, "supplied-reset")
         else:
@@ -286,16 +334,17 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
     del s
     torch.cuda.empty_cache()
     # the workload is defined as a sweep over tau: whole-run updates/s at tau = 1 and 48 too (T = 3)
-    sweep = {str(tau): {v: out["updates_per_s_tau%d_%s" % (tau, v)] for v in ("direct", "fused")}}
+    sweep = {str(tau): {v: out["updates_per_s_tau%d_%s" % (tau, v)] for v in ("direct", "fused", "lazy")}}
     for t_in in (1, 48):
         wt = workloads.workload("stress_tau12", tau=t_in)
         s = SlowMo(wt)
         s.alloc_gradient()
         s.fill_gradient()
         sweep[str(t_in)] = {}
-        for variant in ("direct", "fused"):
+        for variant in ("direct", "fused", "lazy"):
             s.set_variant("outer", variant)
-            total, _, _ = time_steps(s, wt, wt["T"], 1, s.grad, fused=variant == "fused")
+            total, _, _ = time_steps(s, wt, wt["T"], 1, s.grad, fused=variant in ("fused", "lazy"),
+                                     lazy=variant == "lazy")
             sweep[str(t_in)][variant] = wt["m"] * wt["P"] * t_in * wt["T"] / (total * 1e-3)
         s.close()
         del s
@@ -334,8 +383,9 @@ def run_ours(args):
     peak, peak_kind = measured_peak()
     s = SlowMo(w)
     s.set_variant("outer", args.outer_variant)
-    fused = (args.outer_variant == "fused" and (w["grad_mode"] == "supplied" or w["m"] <= 64) and w["tau"] > 1
-             and not w["base"].startswith("sgp"))
+    fused = (args.outer_variant in ("fused", "lazy") and (w["grad_mode"] == "supplied" or w["m"] <= 64)
+             and w["tau"] > 1 and not w["base"].startswith("sgp") and not w.get("no_average"))
+    lazy = fused and args.outer_variant == "lazy"
     grad = None
     if w["grad_mode"] == "supplied":
         grad = s.alloc_gradient()
@@ -343,7 +393,8 @@ def run_ours(args):
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, local_ms, outer_ms = time_steps(s, w, args.steps, args.warmup, grad, fused=fused)
+    total_ms, local_ms, outer_ms = time_steps(s, w, args.steps, args.warmup, grad, fused=fused, lazy=lazy)
+    first_ms = time_steps.first_ms
     clocks = sampler.stop()
     units = w["m"] * w["P"] * w["tau"] * args.steps
     value, ms = aggregate_throughput(units, total_ms, dev)
@@ -374,17 +425,22 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{args.workload}: P={w['P']} m={w['m']} tau={w['tau']} "
                                f"base={w['base']} buffers={w['buffer_policy']} grad={w['grad_mode']}",
-                   "step": ("one outer iteration = tau-1 local-step launches + one launch of the outer step "
+                   "step": ("one outer iteration = tau-1 local-step launches (the first reads the anchor in "
+                            "place of the replica rows) + one launch of the outer step with the last inner "
+                            "step fused in and the broadcast left to the next iteration (SLOWMO_OUTER_LAZY); "
+                            "the timed region ends with slowmo_materialize") if lazy else
+                           ("one outer iteration = tau-1 local-step launches + one launch of the outer step "
                             "with the last inner step fused in (SLOWMO_OUTER_FUSED)") if fused else
                            "one outer iteration = tau local-step launches + one outer-step launch",
                    "outer_variant": args.outer_variant,
                    "replicas": "independent replica of the workload per GPU, no collective on the data path",
                    "l2": "state tensors (>= 5 GB) are far larger than the 126 MB L2; no flush needed"},
-        "gpu_launches": args.steps * (w["tau"] + (0 if fused else 1)),
+        "gpu_launches": args.steps * (w["tau"] + (0 if fused else 1)) + (1 if lazy else 0),
         "clocks": clocks,
         "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
                              w["grad_mode"] if w["base"] == "nesterov" else None),
         "roofline_outer_step": (
+            roofline("last_step_outer", lazy_outer_step_bytes(w), outer_ms, peak, peak_kind) if lazy else
             roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind,
                      f"{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if fused else
             roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
@@ -392,6 +448,9 @@ def run_ours(args):
                      and w["buffer_policy"] != "maintain" else None)),
         "e2e": e2e,
     }
+    if lazy and first_ms is not None:
+        line["roofline_first_local_step"] = roofline("local_step", virtual_first_step_bytes(w), first_ms, peak,
+                                                     peak_kind)
     if rank == 0 and world == 1:
         if not args.no_stress:
             try:
@@ -445,7 +504,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50")
-    ap.add_argument("--outer-variant", default="fused", choices=["direct", "staged", "fused"])
+    ap.add_argument("--outer-variant", default="lazy", choices=["direct", "staged", "fused", "lazy"])
     ap.add_argument("--P", type=int, default=None, help="override the workload's parameter count")
     ap.add_argument("--m", type=int, default=None, help="override the workload's worker count")
     ap.add_argument("--tau", type=int, default=None, help="override the workload's inner steps")

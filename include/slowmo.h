@@ -74,9 +74,16 @@ enum {
   SLOWMO_VARIANT_DEFAULT = 0,
   SLOWMO_OUTER_DIRECT = 1, /* vector loads straight to registers                      */
   SLOWMO_OUTER_STAGED = 2, /* bulk-copy (TMA) staging of row tiles through shared mem  */
-  SLOWMO_OUTER_FUSED = 3   /* the last inner step of each outer iteration runs inside the
+  SLOWMO_OUTER_FUSED = 3,  /* the last inner step of each outer iteration runs inside the
                               outer-step kernel (same results, fewer HBM bytes); see
                               slowmo_local_steps for what this changes for the caller       */
+  SLOWMO_OUTER_LAZY = 4    /* SLOWMO_OUTER_FUSED, and in addition the outer step does not write
+                              the m broadcast rows (nor the reset / averaged buffer rows): the
+                              first inner step of the next iteration reads the anchor (and zero,
+                              or the mean kept in row 0) instead of the rows. Same results through
+                              the API; the caller's raw x, h, v tensors are up to date only after
+                              slowmo_materialize or any call that reads state. Needs tau >= 2,
+                              otherwise it behaves as SLOWMO_OUTER_FUSED                     */
 };
 
 /*
@@ -168,7 +175,8 @@ int slowmo_destroy(slowmo_ctx *ctx);
  * then the caller's x, h, v tensors hold the state before that step, and in supplied mode
  * `grad` must stay valid and unchanged until slowmo_outer_step has been enqueued. Every
  * library call that reads or writes state (slowmo_get_params, slowmo_set_params,
- * slowmo_sync_status, slowmo_set_variant, slowmo_destroy) first runs the deferred step, so
+ * slowmo_sync_status, slowmo_set_variant, slowmo_materialize, slowmo_destroy) first runs the
+ * deferred step, so
  * results seen through the API are the same as without the variant.
  */
 int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad);
@@ -204,6 +212,11 @@ int slowmo_outer_step(slowmo_ctx *ctx);
  * completion before returning.
  */
 int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks);
+
+/* Bring the caller's x, h, v tensors up to date: runs a deferred last inner step
+ * (SLOWMO_OUTER_FUSED) and writes out virtual replicas and buffers (SLOWMO_OUTER_LAZY).
+ * A no-op with the other variants. Enqueued on the stream. */
+int slowmo_materialize(slowmo_ctx *ctx);
 
 /* Change the base learning rate (a schedule's gamma_t). Legal only between outer
  * iterations, i.e. when k = 0 (ESTATE otherwise). EINVAL unless gamma > 0 and finite. */

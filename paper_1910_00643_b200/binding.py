@@ -19,12 +19,12 @@ POLICY = {"reset": 0, "maintain": 1, "average": 2}
 GRAD = {"generated": 0, "supplied": 1}
 TENSOR = {"x": 0, "anchor": 1, "u": 2, "h": 3, "v": 4, "a": 5, "c": 6}
 KERNEL = {"local": 0, "outer": 1}
-VARIANT = {"default": 0, "direct": 1, "staged": 2, "fused": 3}
+VARIANT = {"default": 0, "direct": 1, "staged": 2, "fused": 3, "lazy": 4}
 EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_outer_step",
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
-           "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host"]
+           "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize"]
 
 
 class SlowMoError(RuntimeError):
@@ -81,6 +81,7 @@ def lib():
             "slowmo_last_cuda_error": [vp],
             "slowmo_debug_wait_timeout": [vp, u32],
             "slowmo_iteration_host": [vp, vp, vp, u32],
+            "slowmo_materialize": [vp],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -223,6 +224,9 @@ class SlowMo:
         anchor (torch CPU tensors, pinned for overlap, or numpy arrays)."""
         ptr = lambda a: a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
         _check(lib().slowmo_iteration_host(self.ctx, ptr(c_host), ptr(anchor_host), chunks), "slowmo_iteration_host")
+
+    def materialize(self):
+        _check(lib().slowmo_materialize(self.ctx), "slowmo_materialize")
 
     def set_gamma(self, gamma):
         _check(lib().slowmo_set_gamma(self.ctx, gamma), "slowmo_set_gamma")

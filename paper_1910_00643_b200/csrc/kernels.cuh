@@ -115,6 +115,10 @@ struct LocalArgs {
   float *x, *h, *v;       // [m, pitch]
   const float *src;       // generated mode: centres c [m, pitch]; supplied mode: gradient G [m, pitch]
   const float *a;         // [pitch], generated mode
+  const float *anchor;    // [pitch]: x_{t,0}, read in place of the x rows when the replicas are virtual
+  int virt;               // 0: rows hold the state. Else the outer step left the broadcast (and the buffer
+                          // policy) to this launch: x_i = anchor for every i, and the buffers are
+                          // 1: as stored (maintain), 2: zero (reset), 3: the mean kept in row 0 (average)
   uint64_t pitch;
   uint32_t nvec;          // 4-element column groups per row (of the column window being processed)
   uint32_t vec0;          // index of the window's first column group in the whole vector (noise index)
@@ -213,23 +217,46 @@ local_step_kernel(const LocalArgs A) {
 // and consecutive rows of a thread's loads are independent, so fewer threads keep as many
 // bytes in flight. Same arithmetic per element as local_step_kernel: results are identical.
 // Needs the row keys in the kernel arguments (m <= kInlineKeys) in generated mode.
-template <int BASE, int GRAD, int ROWS>
-__global__ void __launch_bounds__(kThreads)
+#ifndef SLOWMO_VIRT_MIN_BLOCKS
+#define SLOWMO_VIRT_MIN_BLOCKS 4   // resident blocks per SM asked of the virtual-replica form
+#endif
+template <int BASE, int GRAD, int ROWS, bool VIRT>
+__global__ void __launch_bounds__(kThreads, VIRT ? SLOWMO_VIRT_MIN_BLOCKS : 1)
 local_step_cols_kernel(const LocalArgs A) {
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
   if (vi >= A.nvec) return;
   const uint64_t col = 4ull * vi;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
   if (GRAD == 0) a = ld_shared_row(A.a + col);
+  // virtual replicas: every row starts from the anchor; buffers from zero or from the mean in row 0
+  float4 x_all = a, h_all = make_float4(0.f, 0.f, 0.f, 0.f), v_all = h_all;
+  if (VIRT) {
+    x_all = ld_stream(A.anchor + col);
+    if (A.virt == 3) {
+      h_all = ld_stream(A.h + col);
+      if (BASE == 1) v_all = ld_stream(A.v + col);
+    }
+  }
   for (uint32_t i0 = 0; i0 < A.m; i0 += ROWS) {
     float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
 #pragma unroll
     for (int q = 0; q < ROWS; ++q) {
       if (i0 + q < A.m) {
         const uint64_t off = (uint64_t)(i0 + q) * A.pitch + col;
-        x[q] = ld_stream(A.x + off);
-        h[q] = ld_stream(A.h + off);
-        if (BASE == 1) v[q] = ld_stream(A.v + off);
+        if (!VIRT) {
+          x[q] = ld_stream(A.x + off);
+          h[q] = ld_stream(A.h + off);
+          if (BASE == 1) v[q] = ld_stream(A.v + off);
+        } else {
+          x[q] = x_all;
+          if (A.virt == 1) {
+            h[q] = ld_stream(A.h + off);
+            if (BASE == 1) v[q] = ld_stream(A.v + off);
+          } else {
+            h[q] = h_all;
+            v[q] = v_all;
+          }
+        }
         s[q] = ld_stream(A.src + off);
       }
     }
@@ -337,6 +364,33 @@ outer_step_direct_kernel(const OuterArgs A) {
     if (NBUF == 2) {
       const float4 vbar = ordered_row_mean<8>(A.v + col, A.pitch, A.m, A.m_float);
       store_rows(A.v + col, A.pitch, A.m, vbar);
+    }
+  }
+}
+
+// Writes out what a lazy outer step left virtual: x_i = anchor for every row, and the buffer
+// rows per policy (2: zeros, 3: copies of row 0; 1: nothing to do).
+template <int NBUF>
+__global__ void __launch_bounds__(kThreads)
+materialize_kernel(float *x, float *h, float *v, const float *anchor, uint64_t pitch, uint32_t nvec, uint32_t m,
+                   int virt) {
+  const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
+  if (vi >= nvec) return;
+  const uint64_t col = 4ull * vi;
+  const float4 x0 = ld_stream(anchor + col);
+  for (uint32_t i = 0; i < m; ++i) st_stream(x + (uint64_t)i * pitch + col, x0);
+  if (virt == 2) {
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (uint32_t i = 0; i < m; ++i) {
+      st_stream(h + (uint64_t)i * pitch + col, zero);
+      if (NBUF == 2) st_stream(v + (uint64_t)i * pitch + col, zero);
+    }
+  } else if (virt == 3) {
+    const float4 hb = ld_stream(h + col);
+    for (uint32_t i = 1; i < m; ++i) st_stream(h + (uint64_t)i * pitch + col, hb);
+    if (NBUF == 2) {
+      const float4 vb = ld_stream(v + col);
+      for (uint32_t i = 1; i < m; ++i) st_stream(v + (uint64_t)i * pitch + col, vb);
     }
   }
 }

@@ -36,7 +36,10 @@ __device__ __forceinline__ float4 div4(const float4 &s, float d) {
 
 // One thread = one 4-element column group, all m rows. ROWS rows are loaded together.
 // Requires m <= kInlineKeys in generated mode (the launcher falls back otherwise).
-template <int BASE, int GRAD, int POLICY, int ROWS>
+// LAZY: the broadcast and the reset / average of the buffers are left to the next local step
+// (which then reads the anchor instead of the m rows): x rows are not written, "reset" writes
+// nothing, "average" writes the means to row 0 only.
+template <int BASE, int GRAD, int POLICY, int ROWS, bool LAZY>
 __global__ void __launch_bounds__(kThreads, SLOWMO_FUSED_MIN_BLOCKS)
 last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
@@ -103,37 +106,46 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
   }
   st_stream(O.u + col, un);
   st_stream(O.anchor + col, xn);
-  store_rows(O.x + col, O.pitch, m, xn);
+  if (!LAZY) store_rows(O.x + col, O.pitch, m, xn);
   if (POLICY == 0) {
-    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-    store_rows(O.h + col, O.pitch, m, zero);
-    if (BASE == 1) store_rows(O.v + col, O.pitch, m, zero);
+    if (!LAZY) {
+      const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+      store_rows(O.h + col, O.pitch, m, zero);
+      if (BASE == 1) store_rows(O.v + col, O.pitch, m, zero);
+    }
   } else if (POLICY == 2) {
-    store_rows(O.h + col, O.pitch, m, div4(sh, O.m_float));
-    if (BASE == 1) store_rows(O.v + col, O.pitch, m, div4(sv, O.m_float));
+    store_rows(O.h + col, O.pitch, LAZY ? 1u : m, div4(sh, O.m_float));
+    if (BASE == 1) store_rows(O.v + col, O.pitch, LAZY ? 1u : m, div4(sv, O.m_float));
   }
 }
 
-template <int BASE, int GRAD>
+template <int BASE, int GRAD, bool LAZY>
 inline void launch_last_step_outer_policy(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
   const uint32_t blocks = (O.nvec + kThreads - 1) / kThreads;
   constexpr int ROWS = BASE == 1 ? SLOWMO_FUSED_ROWS / 2 : SLOWMO_FUSED_ROWS;
   switch (policy) {
-    case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
-    case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
-    default: last_step_outer_kernel<BASE, GRAD, 2, ROWS><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    default: last_step_outer_kernel<BASE, GRAD, 2, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
+  }
+}
+
+template <bool LAZY>
+inline void launch_last_step_outer_lazy(const LocalArgs &L, const OuterArgs &O, bool adam, bool generated, int policy,
+                                        cudaStream_t stream) {
+  if (adam) {
+    if (generated) launch_last_step_outer_policy<1, 0, LAZY>(L, O, policy, stream);
+    else launch_last_step_outer_policy<1, 1, LAZY>(L, O, policy, stream);
+  } else {
+    if (generated) launch_last_step_outer_policy<0, 0, LAZY>(L, O, policy, stream);
+    else launch_last_step_outer_policy<0, 1, LAZY>(L, O, policy, stream);
   }
 }
 
 inline void launch_last_step_outer(const LocalArgs &L, const OuterArgs &O, bool adam, bool generated, int policy,
-                                   cudaStream_t stream) {
-  if (adam) {
-    if (generated) launch_last_step_outer_policy<1, 0>(L, O, policy, stream);
-    else launch_last_step_outer_policy<1, 1>(L, O, policy, stream);
-  } else {
-    if (generated) launch_last_step_outer_policy<0, 0>(L, O, policy, stream);
-    else launch_last_step_outer_policy<0, 1>(L, O, policy, stream);
-  }
+                                   bool lazy, cudaStream_t stream) {
+  if (lazy) launch_last_step_outer_lazy<true>(L, O, adam, generated, policy, stream);
+  else launch_last_step_outer_lazy<false>(L, O, adam, generated, policy, stream);
 }
 
 }  // namespace slowmo

@@ -32,6 +32,7 @@ struct slowmo_ctx {
   float gamma;               // gamma_t in force
   std::vector<uint64_t> tensor_offsets;  // n_tensors + 1 prefix sums, or empty
   int outer_variant;
+  int virt;                  // lazy variant: 0, or how the next local step must read the (virtual) replicas
   bool pending_last;         // fused variant: the last inner step waits to run inside the outer step
   LocalArgs pending;         // its arguments (counters k, l already include it)
   int *status_dev;           // device status block: [0] = timeout flag, [1] = where
@@ -75,12 +76,21 @@ bool use_column_owner(const slowmo_ctx *ctx) {
   return ctx->cfg.grad_mode == SLOWMO_GRAD_GENERATED;
 }
 
+#ifndef SLOWMO_VIRT_ROWS_DIV
+#define SLOWMO_VIRT_ROWS_DIV 2   // the virtual-replica form keeps ROWS / this many rows in flight
+#endif
 template <int BASE, int GRAD>
 void launch_local(slowmo_ctx *ctx, const LocalArgs &A) {
-  if (use_column_owner(ctx)) {
-    constexpr int ROWS = BASE == 1 ? SLOWMO_LOCAL_COL_ROWS / 2 : SLOWMO_LOCAL_COL_ROWS;
+  constexpr int ROWS = BASE == 1 ? SLOWMO_LOCAL_COL_ROWS / 2 : SLOWMO_LOCAL_COL_ROWS;
+  if (A.virt) {  // first step after a lazy outer step: only the column owner can read virtual replicas
     const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
-    local_step_cols_kernel<BASE, GRAD, ROWS><<<blocks, kThreads, 0, ctx->stream>>>(A);
+    local_step_cols_kernel<BASE, GRAD, (SLOWMO_VIRT_ROWS_DIV > 1 && ROWS > 1) ? ROWS / SLOWMO_VIRT_ROWS_DIV : ROWS, true>
+        <<<blocks, kThreads, 0, ctx->stream>>>(A);
+    return;
+  }
+  if (use_column_owner(ctx)) {
+    const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
+    local_step_cols_kernel<BASE, GRAD, ROWS, false><<<blocks, kThreads, 0, ctx->stream>>>(A);
     return;
   }
   const uint32_t per_tile = kThreads * kLocalUnroll;
@@ -113,10 +123,23 @@ void launch_local_any(slowmo_ctx *ctx, const LocalArgs &A) {
 // Fused variant: run the deferred last inner step on its own (state is about to be read or
 // written from outside).
 int flush_pending(slowmo_ctx *ctx) {
-  if (!ctx->pending_last) return SLOWMO_OK;
-  ctx->pending_last = false;
-  launch_local_any(ctx, ctx->pending);
-  return check_launch(ctx);
+  if (ctx->pending_last) {
+    ctx->pending_last = false;
+    launch_local_any(ctx, ctx->pending);
+    if (int rc = check_launch(ctx)) return rc;
+  }
+  if (ctx->virt) {
+    // lazy variant: write out the virtual replicas and buffers
+    const uint32_t blocks = (ctx->nvec + kThreads - 1) / kThreads;
+    const slowmo_buffers &b = ctx->buf;
+    if (is_adam(ctx->cfg.base))
+      materialize_kernel<2><<<blocks, kThreads, 0, ctx->stream>>>(b.x, b.h, b.v, b.anchor, b.pitch, ctx->nvec, ctx->cfg.m, ctx->virt);
+    else
+      materialize_kernel<1><<<blocks, kThreads, 0, ctx->stream>>>(b.x, b.h, b.v, b.anchor, b.pitch, ctx->nvec, ctx->cfg.m, ctx->virt);
+    ctx->virt = 0;
+    return check_launch(ctx);
+  }
+  return SLOWMO_OK;
 }
 
 // Resolve a tensor id to (base pointer, rows); NULL if the tensor does not exist here.
@@ -217,6 +240,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   ctx->pow_b1 = ctx->pow_b2 = 1.0;
   ctx->gamma = cfg->gamma;
   ctx->outer_variant = SLOWMO_VARIANT_DEFAULT;
+  ctx->virt = 0;
   ctx->pending_last = false;
   ctx->status_dev = nullptr;
   ctx->cuda_error = 0;
@@ -310,6 +334,8 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
   A.v = ctx->buf.v ? ctx->buf.v + woff : nullptr;
   A.src = (generated ? ctx->buf.c : grad) + woff;
   A.a = ctx->buf.a ? ctx->buf.a + woff : nullptr;
+  A.anchor = ctx->buf.anchor + woff;
+  A.virt = 0;
   A.pitch = ctx->buf.pitch;
   A.nvec = ctx->win_nvec;
   A.vec0 = ctx->win_vec0;
@@ -336,10 +362,13 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     A.k = ctx->k;
     if (generated && c.m <= kInlineKeys)
       for (uint32_t i = 0; i < c.m; ++i) A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, i);
+    // lazy variant: the first step of an outer iteration reads the anchor in place of the rows
+    A.virt = ctx->virt;
+    ctx->virt = 0;
     ctx->k += 1;
-    // fused variant: step tau-1 is taken inside the outer-step kernel
-    if (ctx->outer_variant == SLOWMO_OUTER_FUSED && ctx->k == c.tau && (!generated || c.m <= kInlineKeys) &&
-        !is_sgp(c.base) && !c.no_average) {
+    // fused and lazy variants: step tau-1 is taken inside the outer-step kernel
+    if ((ctx->outer_variant == SLOWMO_OUTER_FUSED || ctx->outer_variant == SLOWMO_OUTER_LAZY) && ctx->k == c.tau &&
+        (!generated || c.m <= kInlineKeys) && !is_sgp(c.base) && !c.no_average && A.virt == 0) {
       ctx->pending = A;
       ctx->pending_last = true;
       break;
@@ -375,7 +404,7 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
 
   int variant = ctx->outer_variant;
   if (variant == SLOWMO_VARIANT_DEFAULT) variant = SLOWMO_OUTER_DIRECT;
-  if (ctx->pending_last && variant != SLOWMO_OUTER_FUSED) {
+  if ((ctx->pending_last && variant != SLOWMO_OUTER_FUSED && variant != SLOWMO_OUTER_LAZY) || ctx->virt) {
     if (int rc = flush_pending(ctx)) return rc;
   }
   if (c.no_average) {
@@ -391,8 +420,12 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
     }
   } else if (ctx->pending_last) {
     ctx->pending_last = false;
+    // lazy: leave broadcast and buffer policy to the next local step (needs tau >= 2, so that this
+    // next step is not itself a deferred one)
+    const bool lazy = variant == SLOWMO_OUTER_LAZY && c.tau >= 2;
     launch_last_step_outer(ctx->pending, A, c.base == SLOWMO_BASE_ADAM, c.grad_mode == SLOWMO_GRAD_GENERATED,
-                           c.buffer_policy, ctx->stream);
+                           c.buffer_policy, lazy, ctx->stream);
+    if (lazy) ctx->virt = c.buffer_policy == SLOWMO_BUF_MAINTAIN ? 1 : (c.buffer_policy == SLOWMO_BUF_RESET ? 2 : 3);
   } else if (variant == SLOWMO_OUTER_STAGED) {
     launch_outer_staged(A, nbuf, c.buffer_policy, ctx->num_sms, ctx->status_dev, ctx->stream);
   } else {
@@ -437,6 +470,7 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
 
   const uint64_t t0 = ctx->t, l0 = ctx->l;
   const double p1 = ctx->pow_b1, p2 = ctx->pow_b2;
+  const int virt0 = ctx->virt;
   for (uint32_t w = 0; w < nwin && e == cudaSuccess && rc == SLOWMO_OK; ++w) {
     const uint32_t vec0 = w * win, nv = ctx->nvec - vec0 < win ? ctx->nvec - vec0 : win;
     const uint64_t col0 = 4ull * vec0;
@@ -452,6 +486,7 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
     ctx->l = l0;
     ctx->pow_b1 = p1;
     ctx->pow_b2 = p2;
+    ctx->virt = virt0;
     ctx->win_vec0 = vec0;
     ctx->win_nvec = nv;
     rc = slowmo_local_steps(ctx, c.tau, nullptr);
@@ -471,6 +506,12 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
     if (x) cudaEventDestroy(x);
   if (rc != SLOWMO_OK) return rc;
   return cuda_fail(ctx, e);
+}
+
+int slowmo_materialize(slowmo_ctx *ctx) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  return flush_pending(ctx);
 }
 
 int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t) {
@@ -534,7 +575,7 @@ int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant) {
   if (!ctx) return SLOWMO_EINVAL;
   if (kernel == SLOWMO_K_OUTER) {
     if (variant != SLOWMO_VARIANT_DEFAULT && variant != SLOWMO_OUTER_DIRECT && variant != SLOWMO_OUTER_STAGED &&
-        variant != SLOWMO_OUTER_FUSED)
+        variant != SLOWMO_OUTER_FUSED && variant != SLOWMO_OUTER_LAZY)
       return SLOWMO_EINVAL;
     if (int rc = flush_pending(ctx)) return rc;
     ctx->outer_variant = variant;

@@ -117,7 +117,8 @@ def test_product_code_never_touches_the_oracle():
 
 def test_workload_descriptions():
     from paper_1910_00643_b200 import workloads
-    from bench import fused_outer_step_bytes, local_step_bytes, outer_step_bytes
+    from bench import (fused_outer_step_bytes, lazy_outer_step_bytes, local_step_bytes, outer_step_bytes,
+                       virtual_first_step_bytes)
     w = workloads.workload("resnet50")
     sizes = workloads.tensor_sizes(w["P"], w["n_tensors"], w["seed"])
     assert len(sizes) == 161 and int(sizes.sum()) == w["P"] and sizes.min() >= 1
@@ -138,6 +139,12 @@ def test_workload_descriptions():
     assert fused_outer_step_bytes(ws) / ws["P"] == 96
     assert fused_outer_step_bytes(w) / w["P"] == 20 * 32 + 20
     assert fused_outer_step_bytes(wa) / wa["P"] == 28 * 8 + 20
+    # lazy variant: no broadcast rows, no reset / averaged buffer rows; the next step reads the anchor
+    assert lazy_outer_step_bytes(w) / w["P"] == 12 * 32 + 20 + 4            # average: + one row of means
+    assert virtual_first_step_bytes(w) / w["P"] == 12 * 32 + 8 + 4
+    assert lazy_outer_step_bytes(ws) / ws["P"] == 12 * 4 + 16               # reset, supplied
+    assert virtual_first_step_bytes(ws) / ws["P"] == 12 * 4 + 4
+    assert lazy_outer_step_bytes(wa) / wa["P"] == 16 * 8 + 20 + 8 * 8       # maintain keeps the buffer rows
     j = workloads.sample_coordinates(10**9, 1000, seed=1)
     assert j[0] == 0 and j[-1] == 10**9 - 1 and len(np.unique(j)) == len(j)
 

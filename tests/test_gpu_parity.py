@@ -118,7 +118,7 @@ def test_supplied_gradient_fill_matches_oracle():
 SMALL_P = 3 * 1024 + 37  # several 512- and 1024-column tiles and a ragged tail (not a multiple of 4)
 
 
-@pytest.mark.parametrize("variant", ["direct", "staged", "fused"])
+@pytest.mark.parametrize("variant", ["direct", "staged", "fused", "lazy"])
 @pytest.mark.parametrize("base,policy", list(itertools.product(("nesterov", "adam"), ("reset", "maintain", "average"))))
 @pytest.mark.parametrize("m", [1, 3, 4, 9])
 def test_small_runs_match_oracle(base, policy, m, variant):
@@ -137,7 +137,7 @@ def test_small_runs_match_oracle(base, policy, m, variant):
 @pytest.mark.parametrize("P", [1, 2, 3, 4, 5, 511, 512, 513, 1023, 1024, 1025, 2048 + 4])
 def test_ragged_sizes(P):
     w = workloads.workload("tiny", P=P, m=5, tau=2, T=2, buffer_policy="average")
-    for variant in ("direct", "staged", "fused"):
+    for variant in ("direct", "staged", "fused", "lazy"):
         s = _slowmo(w, guard=64)
         s.set_variant("outer", variant)
         s.run(2)
@@ -156,7 +156,7 @@ def test_tiny_workload_full_run():
 
 def test_many_workers():
     w = workloads.workload("tiny", P=2051, m=32, tau=2, T=2, buffer_policy="average")
-    for variant in ("direct", "staged", "fused"):
+    for variant in ("direct", "staged", "fused", "lazy"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
@@ -190,10 +190,11 @@ def test_runs_are_bit_reproducible():
     import torch
     w = workloads.workload("resnet50", P=200_003, m=8, T=2, n_tensors=0)
     outs = []
-    for variant in ("direct", "staged", "direct", "fused"):
+    for variant in ("direct", "staged", "direct", "fused", "lazy"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
+        s.materialize()      # raw tensors are read below; the lazy and fused variants defer some writes
         s.synchronize()
         outs.append([s.t[k].view(-1, s.pitch)[:, :w["P"]].clone() for k in ("x", "anchor", "u", "h")])
         s.close()
@@ -233,6 +234,45 @@ def test_fused_last_step_is_transparent_through_the_api():
     s.alloc_gradient()
     s.fill_gradient()
     s.run(2, s.grad)
+    _check_against_oracle(s, w2, np.arange(w2["P"]), exact=True)
+    s.close()
+
+
+@pytest.mark.parametrize("base,policy", [("nesterov", "reset"), ("nesterov", "average"), ("nesterov", "maintain"),
+                                         ("adam", "average"), ("adam", "reset")])
+def test_lazy_broadcast_is_transparent_through_the_api(base, policy):
+    import torch
+    w = workloads.workload("tiny", P=3100, m=4, tau=3, T=3, base=base, buffer_policy=policy,
+                           gamma=0.01 if base == "adam" else 0.05, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8)
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", "lazy")
+    s.run(1)
+    # the replicas are virtual now: the raw rows lag, the API does not
+    ref1 = oracle.run(oracle.make_config(**dict(w, T=1)), j0=0, n=w["P"])
+    assert np.array_equal(s.get_params("x").view(np.uint32), ref1["x"].view(np.uint32))   # materialises
+    assert np.array_equal(s.get_params("h").view(np.uint32), ref1["h"].view(np.uint32))
+    s.run(1)                                   # virtual again
+    s.local_steps(1)                           # first step reads the anchor
+    s.local_steps(2)
+    s.outer_step()
+    s.materialize()
+    s.synchronize()
+    x = s.t["x"].view(4, s.pitch)[:, :w["P"]]
+    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())     # raw tensors are up to date
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+    # supplied gradient, and switching the variant while the replicas are virtual
+    w2 = workloads.workload("stress_tau12", P=4100, m=3, tau=2, T=4)
+    s = _slowmo(w2)
+    s.set_variant("outer", "lazy")
+    s.alloc_gradient()
+    s.fill_gradient()
+    s.run(2, s.grad)
+    s.set_variant("outer", "staged")
+    s.run(1, s.grad)
+    s.set_variant("outer", "lazy")
+    s.run(1, s.grad)
     _check_against_oracle(s, w2, np.arange(w2["P"]), exact=True)
     s.close()
 
@@ -441,6 +481,8 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     ("sgp_resnet50", dict(P=12_345, m=5, tau=4), "direct", 5),
     ("tiny", dict(P=7_000, m=3, tau=2, buffer_policy="maintain", no_average=True), "direct", 3),
     ("tiny", dict(P=100, m=2, tau=1), "fused", 8),
+    ("tiny", dict(P=10_007, m=3, tau=3, buffer_policy="average"), "lazy", 3),
+    ("transformer_adam", dict(P=9_001, m=4, tau=2, buffer_policy="reset"), "lazy", 2),
 ])
 def test_pipelined_host_iteration_equals_the_plain_call_sequence(name, over, variant, chunks):
     import torch
@@ -558,7 +600,7 @@ def test_full_size_staged_and_fused_outer_steps_equal_direct():
     import torch
     w = workloads.workload("resnet50", T=2)
     res = []
-    for variant in ("direct", "staged", "fused"):
+    for variant in ("direct", "staged", "fused", "lazy"):
         s = _slowmo(w)
         s.set_variant("outer", variant)
         s.run(2)
