@@ -32,7 +32,9 @@ FALLBACK_HBM_GBS = 6650.0
 # of the kernel as it stands.
 NCU_TRAFFIC_RATIO = {("local_step", "generated"): 0.961, ("local_step", "supplied"): 0.980,
                      ("outer_step", "average"): 0.952, ("outer_step", "reset"): 0.973,
-                     ("last_step_outer", "generated-average"): 0.975, ("last_step_outer", "supplied-reset"): 0.983}
+                     ("last_step_outer", "generated-average"): 0.975, ("last_step_outer", "supplied-reset"): 0.983,
+                     ("last_step_outer", "lazy-generated-average"): 1.001, ("last_step_outer", "lazy-supplied-reset"): 0.994,
+                     ("local_step", "virt-generated-average"): 0.940, ("local_step", "virt-supplied-reset"): 0.970}
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -319,9 +321,10 @@ def stress_extra(peak, peak_kind, tau=12, iters=2):
         total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant in ("fused", "lazy"),
                                          lazy=variant == "lazy")
         if variant == "lazy":
-            out["last_step_outer_lazy"] = roofline("last_step_outer", lazy_outer_step_bytes(w), outer, peak, peak_kind)
+            out["last_step_outer_lazy"] = roofline("last_step_outer", lazy_outer_step_bytes(w), outer, peak, peak_kind,
+                                                   "lazy-supplied-reset")
             out["first_local_step_lazy"] = roofline("local_step", virtual_first_step_bytes(w), time_steps.first_ms,
-                                                    peak, peak_kind)
+                                                    peak, peak_kind, "virt-supplied-reset")
         elif variant == "fused":
             out["last_step_outer_fused"] = roofline("last_step_outer", fused_outer_step_bytes(w), outer, peak,
                                                     peak_kind, "supplied-reset")
@@ -440,7 +443,8 @@ def run_ours(args):
         "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
                              w["grad_mode"] if w["base"] == "nesterov" else None),
         "roofline_outer_step": (
-            roofline("last_step_outer", lazy_outer_step_bytes(w), outer_ms, peak, peak_kind) if lazy else
+            roofline("last_step_outer", lazy_outer_step_bytes(w), outer_ms, peak, peak_kind,
+                     f"lazy-{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if lazy else
             roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind,
                      f"{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if fused else
             roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
@@ -449,8 +453,9 @@ def run_ours(args):
         "e2e": e2e,
     }
     if lazy and first_ms is not None:
-        line["roofline_first_local_step"] = roofline("local_step", virtual_first_step_bytes(w), first_ms, peak,
-                                                     peak_kind)
+        line["roofline_first_local_step"] = roofline(
+            "local_step", virtual_first_step_bytes(w), first_ms, peak, peak_kind,
+            f"virt-{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None)
     if rank == 0 and world == 1:
         if not args.no_stress:
             try:
