@@ -7,31 +7,35 @@
 // stay exactly 1 from their initial value 1 and the de-biased z = x / w is x bit for bit: the
 // kernel carries no w and evaluates the gradient at x.
 //
-// One thread owns a 4-column group of ALL m rows: it walks the rows once doing the local step
-// (same arithmetic as local_step_kernel), keeps each row's x_{k+1/2} in its private column of
-// a shared-memory tile (no thread reads another thread's column, so no barrier), then walks
-// the rows again writing x_i = 1/2 x_{k+1/2,i} + 1/2 x_{k+1/2,i-hops}. HBM traffic is the
-// same 20 (28 for Adam) bytes per update as the communication-free step.
+// One thread owns a 4-column group of ALL m rows (column-owner layout). The mixing
+// x_i = 1/2 x_{k+1/2,i} + 1/2 x_{k+1/2,i-hops} couples row i with row i-hops only, so the
+// thread visits the rows along the cycles of i -> i+hops (gcd(m, hops) cycles of length
+// m / gcd): the half-step value of the previous row of the walk is still in registers when
+// the current row needs it, and the first row of a cycle is closed when the walk returns to
+// it. No shared memory, no second pass; HBM traffic is the same 20 (28 for Adam) bytes per
+// update as the communication-free step.
 #pragma once
 #include "kernels.cuh"
 
 #ifndef SLOWMO_SGP_ROWS
-#define SLOWMO_SGP_ROWS 4       // rows loaded together (Nesterov; Adam uses half)
+#define SLOWMO_SGP_ROWS 2       // rows loaded together (Nesterov; Adam uses half)
 #endif
 
 namespace slowmo {
 constexpr int kSgpRows = SLOWMO_SGP_ROWS;
 
-constexpr uint32_t kSgpMaxWorkers = 64;
+constexpr uint32_t kSgpMaxWorkers = kInlineKeys;  // generated mode needs the row keys in the kernel arguments
 
-inline uint32_t sgp_block_threads(uint32_t m) { return m <= 48 ? 128u : 64u; }  // m * threads * 16 B <= 96 KB
+__device__ __forceinline__ float4 half_sum(const float4 &p, const float4 &q) {
+  return make_float4(__fadd_rn(__fmul_rn(0.5f, p.x), __fmul_rn(0.5f, q.x)), __fadd_rn(__fmul_rn(0.5f, p.y), __fmul_rn(0.5f, q.y)),
+                     __fadd_rn(__fmul_rn(0.5f, p.z), __fmul_rn(0.5f, q.z)), __fadd_rn(__fmul_rn(0.5f, p.w), __fmul_rn(0.5f, q.w)));
+}
 
+// `cycles` = gcd(m, hops), `len` = m / cycles (host-computed); hops < m, or hops = 0 with m = 1.
 template <int BASE, int GRAD, int ROWS>
-__global__ void __launch_bounds__(128)
-sgp_step_kernel(const LocalArgs L, uint32_t hops) {
-  extern __shared__ float4 x_half[];  // [m][blockDim.x]
-  const uint32_t bd = blockDim.x, tid = threadIdx.x;
-  const uint32_t vi = blockIdx.x * bd + tid;
+__global__ void __launch_bounds__(kThreads, 3)
+sgp_step_kernel(const LocalArgs L, uint32_t hops, uint32_t cycles, uint32_t len) {
+  const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
   if (vi >= L.nvec) return;
   const uint64_t col = 4ull * vi;
   const uint32_t m = L.m;
@@ -39,78 +43,83 @@ sgp_step_kernel(const LocalArgs L, uint32_t hops) {
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
   if (GRAD == 0) a = ld_shared_row(L.a + col);
 
-  for (uint32_t i0 = 0; i0 < m; i0 += ROWS) {
-    float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
+  for (uint32_t c = 0; c < cycles; ++c) {
+    // walk the cycle c, c+hops, c+2 hops, ... ; `prev` is x_{k+1/2} of the row visited before
+    float4 first = a, prev = a;
+    uint32_t row = c;
+    for (uint32_t n0 = 0; n0 < len; n0 += ROWS) {
+      float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
+      uint32_t rows[ROWS];
+      uint32_t r = row;
 #pragma unroll
-    for (int q = 0; q < ROWS; ++q) {
-      if (i0 + q < m) {
-        const uint64_t off = (uint64_t)(i0 + q) * L.pitch + col;
-        x[q] = ld_stream(L.x + off);
-        h[q] = ld_stream(L.h + off);
-        if (BASE == 1) v[q] = ld_stream(L.v + off);
-        s[q] = ld_stream(L.src + off);
+      for (int q = 0; q < ROWS; ++q) {
+        rows[q] = r;
+        if (n0 + q < len) {
+          const uint64_t off = (uint64_t)r * L.pitch + col;
+          x[q] = ld_stream(L.x + off);
+          h[q] = ld_stream(L.h + off);
+          if (BASE == 1) v[q] = ld_stream(L.v + off);
+          s[q] = ld_stream(L.src + off);
+        }
+        r += hops;
+        if (r >= m) r -= m;
+      }
+      row = r;
+#pragma unroll
+      for (int q = 0; q < ROWS; ++q) {
+        if (n0 + q >= len) break;
+        const uint32_t i = rows[q];
+        float4 g;
+        if (GRAD == 0) {
+          const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * (L.vec0 + vi) + 1);
+          float4 z;
+          word_to_normal_pair(mix64(st), z.x, z.y);
+          word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(L.sigma, comp(z, e)));
+        } else {
+          g = s[q];
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
+        const uint64_t off = (uint64_t)i * L.pitch + col;
+        st_stream(L.h + off, h[q]);
+        if (BASE == 1) st_stream(L.v + off, v[q]);
+        if (n0 + q == 0) {
+          first = x[q];  // its in-neighbour is the last row of the walk
+        } else {
+          st_stream(L.x + off, half_sum(x[q], prev));  // keep half, receive half from the row hops back
+        }
+        prev = x[q];
       }
     }
-#pragma unroll
-    for (int q = 0; q < ROWS; ++q) {
-      const uint32_t i = i0 + q;
-      if (i >= m) break;
-      float4 g;
-      if (GRAD == 0) {
-        const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * (L.vec0 + vi) + 1);
-        float4 z;
-        word_to_normal_pair(mix64(st), z.x, z.y);
-        word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(L.sigma, comp(z, e)));
-      } else {
-        g = s[q];
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
-      const uint64_t off = (uint64_t)i * L.pitch + col;
-      st_stream(L.h + off, h[q]);
-      if (BASE == 1) st_stream(L.v + off, v[q]);
-      x_half[i * bd + tid] = x[q];
-    }
-  }
-
-  // push-sum mixing: keep half, receive half from the worker `hops` places back
-  const uint32_t back = m - hops % m;
-  for (uint32_t i = 0; i < m; ++i) {
-    const uint32_t from = (i + back) % m;
-    const float4 own = x_half[i * bd + tid], got = x_half[from * bd + tid];
-    float4 xn;
-    xn.x = __fadd_rn(__fmul_rn(0.5f, own.x), __fmul_rn(0.5f, got.x));
-    xn.y = __fadd_rn(__fmul_rn(0.5f, own.y), __fmul_rn(0.5f, got.y));
-    xn.z = __fadd_rn(__fmul_rn(0.5f, own.z), __fmul_rn(0.5f, got.z));
-    xn.w = __fadd_rn(__fmul_rn(0.5f, own.w), __fmul_rn(0.5f, got.w));
-    st_stream(L.x + (uint64_t)i * L.pitch + col, xn);
+    st_stream(L.x + (uint64_t)c * L.pitch + col, half_sum(first, prev));
   }
 }
 
-inline cudaError_t sgp_configure() {
-  const int bytes = 96 * 1024;
-  cudaError_t e = cudaSuccess;
-#define SLOWMO_SET(B, G, R)                                                                             \
-  if (e == cudaSuccess)                                                                                 \
-    e = cudaFuncSetAttribute(sgp_step_kernel<B, G, R>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-  SLOWMO_SET(0, 0, kSgpRows) SLOWMO_SET(0, 1, kSgpRows) SLOWMO_SET(1, 0, kSgpRows / 2) SLOWMO_SET(1, 1, kSgpRows / 2)
-#undef SLOWMO_SET
-  return e;
+inline cudaError_t sgp_configure() { return cudaSuccess; }
+
+inline uint32_t sgp_gcd(uint32_t p, uint32_t q) {
+  while (q) {
+    const uint32_t t = p % q;
+    p = q;
+    q = t;
+  }
+  return p;
 }
 
 inline void launch_sgp_step(const LocalArgs &L, uint32_t hops, bool adam, bool generated, cudaStream_t stream) {
-  const uint32_t bd = sgp_block_threads(L.m);
-  const uint32_t blocks = (L.nvec + bd - 1) / bd;
-  const size_t smem = (size_t)L.m * bd * sizeof(float4);
+  const uint32_t blocks = (L.nvec + kThreads - 1) / kThreads;
+  hops = L.m > 1 ? hops % L.m : 0;
+  const uint32_t cycles = hops ? sgp_gcd(L.m, hops) : L.m;  // hops = 0: every row is its own cycle (x unchanged)
+  const uint32_t len = L.m / cycles;
   if (adam) {
-    if (generated) sgp_step_kernel<1, 0, kSgpRows / 2><<<blocks, bd, smem, stream>>>(L, hops);
-    else sgp_step_kernel<1, 1, kSgpRows / 2><<<blocks, bd, smem, stream>>>(L, hops);
+    if (generated) sgp_step_kernel<1, 0, kSgpRows / 2><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else sgp_step_kernel<1, 1, kSgpRows / 2><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
   } else {
-    if (generated) sgp_step_kernel<0, 0, kSgpRows><<<blocks, bd, smem, stream>>>(L, hops);
-    else sgp_step_kernel<0, 1, kSgpRows><<<blocks, bd, smem, stream>>>(L, hops);
+    if (generated) sgp_step_kernel<0, 0, kSgpRows><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else sgp_step_kernel<0, 1, kSgpRows><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
   }
 }
 
