@@ -116,6 +116,9 @@ typedef struct {
                                      that skips the exact average: every worker applies Eq. (2), (3) to
                                      its own x_{t,tau}; anchor and u are then [m, pitch], one row per
                                      worker, and SLOWMO_BUF_AVERAGE is refused (EINVAL)                */
+  uint32_t worker_offset;         /* global index of this context's first worker: row i is worker
+                                     worker_offset + i for the noise and centre streams. 0 unless the m
+                                     workers of a job are spread over several contexts (several GPUs)     */
 } slowmo_config;
 
 /* Device tensors borrowed from the caller (see "Layout" above). */
@@ -212,6 +215,44 @@ int slowmo_outer_step(slowmo_ctx *ctx);
  * completion before returning.
  */
 int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks);
+
+/*
+ * Outer step of Algorithm 1 for workers sharded over several GPUs of one node: the exact average
+ * (the paper's AllReduce) fused with Eq. (2), Eq. (3), the broadcast and the buffer policy in
+ * one kernel per GPU that reads and writes the other GPUs' memory directly.
+ *
+ * GPU r (0 <= r < world <= 16) holds the rows of global workers r*m_local .. r*m_local+m_local-1
+ * in x[r], h[r] (v[r] for Adam bases), each [m_local, pitch], and full [pitch] copies anchor[r],
+ * u[r] of the outer iterate and the slow momentum; the arrays x, h, v, anchor, u are HOST arrays
+ * of `world` device pointers valid on the calling GPU (peer-mapped). The call made on GPU `rank`
+ * handles that GPU's contiguous slice of the columns: it adds the rows of all GPUs in global
+ * worker order (so the result is bit-identical to slowmo_outer_step on one GPU holding all
+ * world*m_local workers), updates u and the anchor, and stores the slice into every GPU's
+ * copies and rows, with the buffer policy. Every GPU makes the call with the same arguments
+ * except `rank`.
+ * Ordering is the caller's: all GPUs' local steps must have finished before any of these
+ * kernels starts, and all of these kernels before anyone's next local step (for instance a
+ * stream-ordered collective on each GPU's stream before and after). The kernels themselves
+ * never wait for one another. Contexts that ran the local steps are told with
+ * slowmo_outer_step_external. The local steps of sharded workers must use a communication-free
+ * base (the SGP bases mix only the rows of one context). Errors as for slowmo_outer_step_static.
+ */
+typedef struct {
+  uint32_t world, rank;
+  uint32_t m_local;              /* workers (rows) per GPU; m = world * m_local                     */
+  uint64_t P, pitch;
+  float *const *x, *const *h, *const *v;  /* [world] device pointers each; v may be NULL for Nesterov bases */
+  float *const *anchor, *const *u;         /* [world] device pointers to the [pitch] copies                  */
+  int32_t base, buffer_policy;   /* SLOWMO_BASE_* (tells whether v exists), SLOWMO_BUF_*             */
+  float alpha, beta, gamma_t;
+} slowmo_shard_args;
+int slowmo_outer_step_sharded(const slowmo_shard_args *args, void *cuda_stream);
+
+/* Tell a context that the outer step of the current iteration was carried out on its tensors by
+ * other means (slowmo_outer_step_sharded): legal after exactly tau local steps (ESTATE
+ * otherwise); runs a deferred last step if there is one, advances t, sets k = 0 and, under the
+ * reset policy, restarts the Adam count. Launches nothing else. */
+int slowmo_outer_step_external(slowmo_ctx *ctx);
 
 /* Bring the caller's x, h, v tensors up to date: runs a deferred last inner step
  * (SLOWMO_OUTER_FUSED) and writes out virtual replicas and buffers (SLOWMO_OUTER_LAZY).

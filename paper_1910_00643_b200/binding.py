@@ -24,7 +24,8 @@ EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_oute
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
-           "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize"]
+           "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize",
+           "slowmo_outer_step_sharded", "slowmo_outer_step_external"]
 
 
 class SlowMoError(RuntimeError):
@@ -44,12 +45,22 @@ class Config(C.Structure):
         ("a_lo", C.c_float), ("a_hi", C.c_float), ("c_std", C.c_float), ("sigma", C.c_float),
         ("x_init", C.c_float),
         ("n_tensors", C.c_uint32), ("tensor_sizes", C.POINTER(C.c_uint64)), ("no_average", C.c_int32),
+        ("worker_offset", C.c_uint32),
     ]
 
 
 class Buffers(C.Structure):
     _fields_ = [("x", C.c_void_p), ("h", C.c_void_p), ("v", C.c_void_p), ("anchor", C.c_void_p),
                 ("u", C.c_void_p), ("a", C.c_void_p), ("c", C.c_void_p), ("pitch", C.c_uint64)]
+
+
+class ShardArgs(C.Structure):
+    _fields_ = [("world", C.c_uint32), ("rank", C.c_uint32), ("m_local", C.c_uint32),
+                ("P", C.c_uint64), ("pitch", C.c_uint64),
+                ("x", C.POINTER(C.c_void_p)), ("h", C.POINTER(C.c_void_p)), ("v", C.POINTER(C.c_void_p)),
+                ("anchor", C.POINTER(C.c_void_p)), ("u", C.POINTER(C.c_void_p)),
+                ("base", C.c_int32), ("buffer_policy", C.c_int32),
+                ("alpha", C.c_float), ("beta", C.c_float), ("gamma_t", C.c_float)]
 
 
 _lib = None
@@ -82,6 +93,8 @@ def lib():
             "slowmo_debug_wait_timeout": [vp, u32],
             "slowmo_iteration_host": [vp, vp, vp, u32],
             "slowmo_materialize": [vp],
+            "slowmo_outer_step_sharded": [C.POINTER(ShardArgs), vp],
+            "slowmo_outer_step_external": [vp],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -107,13 +120,13 @@ def _check(status, what):
 def make_config(*, P, m, tau, alpha=1.0, beta=0.0, gamma=0.1, base="nesterov", mu=0.0, weight_decay=0.0,
                 adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8, buffer_policy="reset", grad_mode="generated",
                 seed=0, a_lo=0.5, a_hi=2.0, c_std=1.0, sigma=0.0, x_init=0.0, tensor_sizes=None, no_average=False,
-                **_ignored):
+                worker_offset=0, **_ignored):
     """Fill the C config from paper-notation keyword arguments (see include/slowmo.h)."""
     cfg = Config(P, m, tau, alpha, beta, gamma, BASE[base] if isinstance(base, str) else base, mu,
                  weight_decay, adam_b1, adam_b2, adam_eps,
                  POLICY[buffer_policy] if isinstance(buffer_policy, str) else buffer_policy,
                  GRAD[grad_mode] if isinstance(grad_mode, str) else grad_mode, seed, a_lo, a_hi, c_std,
-                 sigma, x_init, 0, None, 1 if no_average else 0)
+                 sigma, x_init, 0, None, 1 if no_average else 0, worker_offset)
     if tensor_sizes is not None:
         arr = (C.c_uint64 * len(tensor_sizes))(*[int(s) for s in tensor_sizes])
         cfg._keep = arr
@@ -135,6 +148,22 @@ def outer_step_static(x, h, v, anchor, u, *, pitch, P, m, base, buffer_policy, a
     _check(rc, "slowmo_outer_step_static")
 
 
+def outer_step_sharded(rank, x, h, v, anchor, u, *, m_local, P, pitch, base, buffer_policy, alpha, beta, gamma,
+                       stream=None):
+    """slowmo_outer_step_sharded for GPU `rank`: x, h, v, anchor, u are lists (one entry per GPU) of
+    device pointers (ints) or torch tensors, valid on the calling GPU."""
+    world = len(x)
+    ptr = lambda t: t if isinstance(t, int) or t is None else t.data_ptr()
+    arr = lambda lst: None if lst is None else (C.c_void_p * world)(*[ptr(t) for t in lst])
+    keep = [arr(x), arr(h), arr(v), arr(anchor), arr(u)]
+    cast = lambda a: None if a is None else C.cast(a, C.POINTER(C.c_void_p))
+    args = ShardArgs(world, rank, m_local, P, pitch, cast(keep[0]), cast(keep[1]), cast(keep[2]), cast(keep[3]),
+                     cast(keep[4]), BASE[base] if isinstance(base, str) else base,
+                     POLICY[buffer_policy] if isinstance(buffer_policy, str) else buffer_policy, alpha, beta, gamma)
+    _check(lib().slowmo_outer_step_sharded(C.byref(args), None if stream is None else stream.cuda_stream),
+           "slowmo_outer_step_sharded")
+
+
 def round_up(n, q):
     return (n + q - 1) // q * q
 
@@ -146,7 +175,7 @@ class SlowMo:
     marshal arguments.
     """
 
-    def __init__(self, workload, stream=None, pitch=None, guard=0):
+    def __init__(self, workload, stream=None, pitch=None, guard=0, tensors=None):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("libslowmo needs a CUDA device (sm_100a); there is no CPU path")
@@ -165,6 +194,7 @@ class SlowMo:
         generated = self.cfg.grad_mode == GRAD["generated"]
         self._raw = {}
         self.t = {}
+        self._given = tensors or {}   # caller-allocated tensors (e.g. peer-mapped memory), by name
         self.outer_rows = self.m if self.cfg.no_average else 1
         for name, rows, need in (("x", self.m, True), ("h", self.m, True), ("v", self.m, adam),
                                  ("anchor", self.outer_rows, True), ("u", self.outer_rows, True),
@@ -186,6 +216,10 @@ class SlowMo:
     def _alloc(self, name, rows):
         torch = self.torch
         n = rows * self.pitch
+        if name in self._given:
+            t = self._given[name]
+            assert t.is_cuda and t.dtype == torch.float32 and t.numel() >= n and t.data_ptr() % 16 == 0, name
+            return t.view(-1)[:n]
         g = self.guard
         raw = torch.empty(n + 2 * g, dtype=torch.float32, device="cuda")
         if g:
@@ -224,6 +258,9 @@ class SlowMo:
         anchor (torch CPU tensors, pinned for overlap, or numpy arrays)."""
         ptr = lambda a: a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
         _check(lib().slowmo_iteration_host(self.ctx, ptr(c_host), ptr(anchor_host), chunks), "slowmo_iteration_host")
+
+    def outer_step_external(self):
+        _check(lib().slowmo_outer_step_external(self.ctx), "slowmo_outer_step_external")
 
     def materialize(self):
         _check(lib().slowmo_materialize(self.ctx), "slowmo_materialize")

@@ -55,9 +55,10 @@ __device__ __forceinline__ float comp(const float4 &v, int e) { return reinterpr
 
 // dst[i, j] = scale * z(tag, seed, 0, 0, i, j) for every row i and column j < 4*nvec.
 __global__ void __launch_bounds__(kThreads)
-fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t tag, uint64_t seed, float scale) {
+fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t tag, uint64_t seed, float scale,
+                        uint32_t worker0) {
   const uint32_t row = blockIdx.y;
-  const uint64_t key = stream_key(tag, seed, 0, 0, row);
+  const uint64_t key = stream_key(tag, seed, 0, 0, worker0 + row);  // row i holds global worker worker0 + i
   float *p = dst + (uint64_t)row * pitch;
   for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
     // columns 4vi..4vi+3 are the pairs 2vi and 2vi+1 of the row's stream
@@ -123,6 +124,7 @@ struct LocalArgs {
   uint32_t nvec;          // 4-element column groups per row (of the column window being processed)
   uint32_t vec0;          // index of the window's first column group in the whole vector (noise index)
   uint32_t m;
+  uint32_t worker0;       // global index of row 0's worker (non-zero when the workers are sharded over GPUs)
   uint64_t seed, t;       // outer iteration, for the noise key
   uint32_t k;             // inner step, for the noise key
   float neg_gamma, mu, wd, sigma;
@@ -181,7 +183,7 @@ local_step_kernel(const LocalArgs A) {
     if (A.m <= kInlineKeys) {
       key = A.keys[row];
     } else {  // many workers: one lane per warp derives the key while the loads are in flight
-      if ((threadIdx.x & 31u) == 0) key = stream_key(kTagGradNoise, A.seed, A.t, A.k, row);
+      if ((threadIdx.x & 31u) == 0) key = stream_key(kTagGradNoise, A.seed, A.t, A.k, A.worker0 + row);
       key = __shfl_sync(0xFFFFFFFFu, key, 0);
     }
   }

@@ -13,6 +13,7 @@
 
 #include "kernels.cuh"
 #include "outer_fused.cuh"
+#include "outer_sharded.cuh"
 #include "outer_staged.cuh"
 #include "sgp_step.cuh"
 
@@ -295,7 +296,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   if (e == cudaSuccess && generated) {
     fill_curvature_kernel<<<fill_blocks(ctx, 1), kThreads, 0, ctx->stream>>>(buf->a, ctx->nvec, cfg->seed, cfg->a_lo, cfg->a_hi);
     fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->c, buf->pitch, ctx->nvec, kTagCentre,
-                                                                                   cfg->seed, cfg->c_std);
+                                                                                   cfg->seed, cfg->c_std, cfg->worker_offset);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) {
@@ -340,6 +341,7 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
   A.nvec = ctx->win_nvec;
   A.vec0 = ctx->win_vec0;
   A.m = c.m;
+  A.worker0 = c.worker_offset;
   A.seed = c.seed;
   A.neg_gamma = -ctx->gamma;
   A.mu = c.mu;
@@ -361,7 +363,8 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     A.t = ctx->t;
     A.k = ctx->k;
     if (generated && c.m <= kInlineKeys)
-      for (uint32_t i = 0; i < c.m; ++i) A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, i);
+      for (uint32_t i = 0; i < c.m; ++i)
+        A.keys[i] = stream_key(kTagGradNoise, c.seed, ctx->t, ctx->k, c.worker_offset + i);
     // lazy variant: the first step of an outer iteration reads the anchor in place of the rows
     A.virt = ctx->virt;
     ctx->virt = 0;
@@ -508,6 +511,57 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
   return cuda_fail(ctx, e);
 }
 
+int slowmo_outer_step_external(slowmo_ctx *ctx) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  if (ctx->k != ctx->cfg.tau) return SLOWMO_ESTATE;
+  if (int rc = flush_pending(ctx)) return rc;  // a deferred last step must have run before the rows are used
+  ctx->t += 1;
+  ctx->k = 0;
+  if (ctx->cfg.buffer_policy == SLOWMO_BUF_RESET) {
+    ctx->l = 0;
+    ctx->pow_b1 = ctx->pow_b2 = 1.0;
+  }
+  return SLOWMO_OK;
+}
+
+int slowmo_outer_step_sharded(const slowmo_shard_args *a, void *cuda_stream) {
+  if (!a) return SLOWMO_EINVAL;
+  const bool adam = a->base == SLOWMO_BASE_ADAM || a->base == SLOWMO_BASE_SGP_ADAM;
+  if (a->base < SLOWMO_BASE_NESTEROV || a->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
+  if (a->buffer_policy < SLOWMO_BUF_RESET || a->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
+  if (a->world == 0 || a->world > kMaxShardGpus || a->rank >= a->world || a->m_local == 0) return SLOWMO_EINVAL;
+  if (a->P == 0 || a->P > (1ull << 32) - 4096 || a->pitch < a->P) return SLOWMO_EINVAL;
+  if (a->pitch % 4 != 0) return SLOWMO_EALIGN;
+  if (!finite_pos(a->alpha) || !unit_interval(a->beta) || !finite_pos(a->gamma_t)) return SLOWMO_EINVAL;
+  if (!a->x || !a->h || !a->anchor || !a->u || (adam && !a->v)) return SLOWMO_EINVAL;
+  ShardArgs A;
+  for (uint32_t r = 0; r < a->world; ++r) {
+    A.x[r] = a->x[r];
+    A.h[r] = a->h[r];
+    A.v[r] = adam ? a->v[r] : nullptr;
+    A.anchor[r] = a->anchor[r];
+    A.u[r] = a->u[r];
+    const void *ptrs[] = {A.x[r], A.h[r], A.anchor[r], A.u[r]};
+    for (const void *p : ptrs) {
+      if (!p) return SLOWMO_EINVAL;
+      if (!aligned16(p)) return SLOWMO_EALIGN;
+    }
+    if (adam && (!A.v[r] || !aligned16(A.v[r]))) return A.v[r] ? SLOWMO_EALIGN : SLOWMO_EINVAL;
+  }
+  A.pitch = a->pitch;
+  A.world = a->world;
+  A.rank = a->rank;
+  A.m_local = a->m_local;
+  shard_slice((uint32_t)((a->P + 3) / 4), a->world, a->rank, &A.vec_begin, &A.vec_end);
+  A.beta = a->beta;
+  A.inv_gamma = (float)(1.0 / (double)a->gamma_t);
+  A.neg_alpha_gamma = -(float)((double)a->alpha * (double)a->gamma_t);
+  A.m_float = (float)((uint64_t)a->world * a->m_local);
+  launch_outer_sharded(A, adam ? 2 : 1, a->buffer_policy, (cudaStream_t)cuda_stream);
+  return cudaGetLastError() == cudaSuccess ? SLOWMO_OK : SLOWMO_ECUDA;
+}
+
 int slowmo_materialize(slowmo_ctx *ctx) {
   if (!ctx) return SLOWMO_EINVAL;
   if (ctx->cuda_error) return SLOWMO_ECUDA;
@@ -545,7 +599,7 @@ int slowmo_fill_gradient(slowmo_ctx *ctx, float *grad) {
   if (ctx->cuda_error) return SLOWMO_ECUDA;
   const uint32_t m = ctx->cfg.m;
   fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(
-      grad, ctx->buf.pitch, ctx->nvec, kTagSupplied, ctx->cfg.seed, ctx->cfg.sigma);
+      grad, ctx->buf.pitch, ctx->nvec, kTagSupplied, ctx->cfg.seed, ctx->cfg.sigma, ctx->cfg.worker_offset);
   return check_launch(ctx);
 }
 
