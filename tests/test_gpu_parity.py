@@ -579,16 +579,18 @@ def test_full_size_generated_workloads_on_sampled_coordinates(name):
     torch.cuda.empty_cache()
 
 
-@pytest.mark.parametrize("name", ["stress_tau1", "stress_tau12"])
-def test_full_size_supplied_gradient_on_sampled_coordinates(name):
+@pytest.mark.parametrize("name,variant", [("stress_tau1", "direct"), ("stress_tau12", "direct"),
+                                          ("stress_tau12", "lazy"), ("stress_tau1", "fused")])
+def test_full_size_supplied_gradient_on_sampled_coordinates(name, variant):
     import torch
     w = workloads.workload(name)
     s = _slowmo(w)
+    s.set_variant("outer", variant)
     s.alloc_gradient()
     s.fill_gradient()
     s.run(w["T"], s.grad)
     j = workloads.sample_coordinates(w["P"], 1 << 13, seed=2)
-    _check_against_oracle(s, w, j, exact=True)
+    _check_against_oracle(s, w, j, exact=True)       # reads through sync_status, which writes out lazy state
     x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
     assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
     s.close()
