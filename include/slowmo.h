@@ -293,6 +293,11 @@ int slowmo_fill_gradient(slowmo_ctx *ctx, float *grad);
 int slowmo_debug_noise(slowmo_ctx *ctx, uint32_t tag, uint64_t t, uint32_t k, uint32_t w, uint64_t j0,
                        uint64_t n, uint64_t *words, float *normals);
 
+/* Test hook: the two Box-Muller normals of each of n arbitrary 64-bit words (device arrays):
+ * out[2i] (cosine output) and out[2i+1] (sine output) from words[i]. Lets a test sweep every
+ * value of the 24-bit radius field and of the 24-bit angle field. */
+int slowmo_debug_words_to_normals(slowmo_ctx *ctx, const uint64_t *words, uint64_t n, float *out);
+
 /* Segment idx of the optional parameter-tensor table: first coordinate and length. */
 int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_t *count);
 

@@ -46,6 +46,8 @@ def lib():
         L.oracle_word_to_unit.argtypes = [C.c_uint64]
         L.oracle_word_to_normal_pair.restype = None
         L.oracle_word_to_normal_pair.argtypes = [C.c_uint64, C.POINTER(C.c_float * 2)]
+        L.oracle_words_to_normals.restype = None
+        L.oracle_words_to_normals.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
         L.oracle_stream_normal.restype = C.c_float
         L.oracle_stream_normal.argtypes = [C.c_uint64, C.c_uint64]
         L.oracle_stream_export.restype = None
@@ -122,6 +124,14 @@ def normal_pair(word):
     z = (C.c_float * 2)()
     lib().oracle_word_to_normal_pair(word, C.byref(z))
     return float(z[0]), float(z[1])
+
+
+def words_to_normals(words):
+    """Both Box-Muller normals of every word: float32 array [n, 2]."""
+    words = np.ascontiguousarray(words, dtype=np.uint64)
+    out = np.empty((words.size, 2), np.float32)
+    lib().oracle_words_to_normals(_ptr(words), words.size, _ptr(out))
+    return out
 
 
 def stream(tag, seed, t, k, w, j0, n, words=True, normals=True):

@@ -148,6 +148,11 @@ float oracle_stream_normal(uint64_t key, uint64_t j) {
   return z[j & 1];
 }
 
+/* Bulk form of oracle_word_to_normal_pair for tests: out[2i], out[2i+1] from words[i]. */
+void oracle_words_to_normals(const uint64_t *words, uint64_t n, float *out) {
+  for (uint64_t i = 0; i < n; ++i) oracle_word_to_normal_pair(words[i], out + 2 * i);
+}
+
 void oracle_stream_export(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, uint32_t w,
                           uint64_t j0, uint64_t n, uint64_t *words, float *normals) {
   uint64_t key = oracle_stream_key(tag, seed, t, k, w);

@@ -48,6 +48,7 @@ uint64_t oracle_stream_key(uint32_t tag, uint64_t seed, uint64_t t, uint32_t k, 
 float oracle_word_to_unit(uint64_t r);
 /* Two independent N(0,1) draws from one word: Box-Muller (cosine, sine), binary32 arithmetic. */
 void oracle_word_to_normal_pair(uint64_t r, float z[2]);
+void oracle_words_to_normals(const uint64_t *words, uint64_t n, float *out); /* out[2i], out[2i+1] from words[i] */
 /* Normal of coordinate j in a stream: output (j & 1) of the pair made from word j >> 1. */
 float oracle_stream_normal(uint64_t key, uint64_t j);
 /* Bulk export for tests, for j0 <= j < j0 + n: words[i] = word j0+i of the stream,

@@ -25,7 +25,8 @@ EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_oute
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
            "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize",
-           "slowmo_outer_step_sharded", "slowmo_outer_step_external"]
+           "slowmo_outer_step_sharded", "slowmo_outer_step_external",
+           "slowmo_debug_words_to_normals"]
 
 
 class SlowMoError(RuntimeError):
@@ -95,6 +96,7 @@ def lib():
             "slowmo_materialize": [vp],
             "slowmo_outer_step_sharded": [C.POINTER(ShardArgs), vp],
             "slowmo_outer_step_external": [vp],
+            "slowmo_debug_words_to_normals": [vp, vp, u64, vp],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -320,6 +322,17 @@ class SlowMo:
                                         z.data_ptr() if normals else None), "slowmo_debug_noise")
         self.synchronize()
         return (wd.cpu().numpy().view(np.uint64) if words else None, z.cpu().numpy() if normals else None)
+
+    def debug_words_to_normals(self, words):
+        """Both normals of each 64-bit word (numpy uint64 array) -> float32 [n, 2]."""
+        torch = self.torch
+        w = torch.from_numpy(np.ascontiguousarray(words, dtype=np.uint64).view(np.int64)).cuda()
+        out = torch.empty(2 * w.numel(), dtype=torch.float32, device="cuda")
+        self.stream.wait_stream(torch.cuda.current_stream())
+        _check(lib().slowmo_debug_words_to_normals(self.ctx, w.data_ptr(), w.numel(), out.data_ptr()),
+               "slowmo_debug_words_to_normals")
+        self.synchronize()
+        return out.cpu().numpy().reshape(-1, 2)
 
     def tensor_range(self, idx):
         off, cnt = C.c_uint64(), C.c_uint64()

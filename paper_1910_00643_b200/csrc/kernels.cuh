@@ -108,6 +108,17 @@ export_stream_kernel(uint64_t key, uint64_t j0, uint64_t n, uint64_t *words, flo
   }
 }
 
+// Test hook: both normals of arbitrary words, out[2i], out[2i+1] from words[i].
+__global__ void __launch_bounds__(kThreads)
+words_to_normals_kernel(const uint64_t *words, uint64_t n, float *out) {
+  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (uint64_t)gridDim.x * kThreads) {
+    float zc, zs;
+    word_to_normal_pair(words[i], zc, zs);
+    out[2 * i] = zc;
+    out[2 * i + 1] = zs;
+  }
+}
+
 // ---- K1: fused multi-replica base-optimizer step ------------------------------------------
 
 constexpr uint32_t kInlineKeys = 64;  // noise keys of up to this many rows travel in the kernel arguments

@@ -617,6 +617,17 @@ int slowmo_debug_noise(slowmo_ctx *ctx, uint32_t tag, uint64_t t, uint32_t k, ui
   return check_launch(ctx);
 }
 
+int slowmo_debug_words_to_normals(slowmo_ctx *ctx, const uint64_t *words, uint64_t n, float *out) {
+  if (!ctx || (n && (!words || !out))) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  if (n == 0) return SLOWMO_OK;
+  uint64_t blocks = (n + kThreads - 1) / kThreads;
+  const uint64_t cap = (uint64_t)ctx->num_sms * 16;
+  if (blocks > cap) blocks = cap;
+  words_to_normals_kernel<<<(uint32_t)blocks, kThreads, 0, ctx->stream>>>(words, n, out);
+  return check_launch(ctx);
+}
+
 int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_t *count) {
   if (!ctx || !offset || !count) return SLOWMO_EINVAL;
   if (ctx->tensor_offsets.empty() || idx >= ctx->cfg.n_tensors) return SLOWMO_EINVAL;

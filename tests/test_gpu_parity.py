@@ -82,6 +82,21 @@ def test_normals_bit_exact_on_a_large_sample():
     s.close()
 
 
+def test_normal_map_is_bit_exact_for_every_radius_field_and_every_angle_field():
+    # z = radius(k1) * trig(k2) with an IEEE multiply, so agreement for all 2^24 values of each field
+    # (with the other field fixed) gives agreement for every word
+    s = _slowmo(workloads.workload("tiny"))
+    all24 = np.arange(1 << 24, dtype=np.uint64)
+    for words in (all24 << np.uint64(40),                                   # every k1, angle 0: zc = radius
+                  (all24 << np.uint64(40)) | np.uint64(0x1234560000),       # every k1, a generic angle
+                  all24 << np.uint64(16),                                   # every k2, largest radius
+                  (np.uint64(0x5A5A5A) << np.uint64(40)) | (all24 << np.uint64(16)) | np.uint64(0xBEEF)):
+        got = s.debug_words_to_normals(words)
+        ref = oracle.words_to_normals(words)
+        assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+    s.close()
+
+
 def test_problem_data_fill_matches_oracle():
     w = workloads.workload("tiny", P=5003, m=3, a_lo=0.1, a_hi=1.0, c_std=0.05, seed=5)
     s = _slowmo(w, guard=64)

@@ -104,6 +104,15 @@ def test_normal_map_against_double_precision_box_muller():
     assert np.abs(z).max() <= math.sqrt(2 * 24 * math.log(2)) + 1e-5
 
 
+def test_normal_map_against_libm_for_every_radius_field_and_every_angle_field():
+    # exhaustive in each 24-bit field of the word (the other one fixed)
+    all24 = np.arange(1 << 24, dtype=np.uint64)
+    for words in (all24 << np.uint64(40), (np.uint64(0x000100) << np.uint64(40)) | (all24 << np.uint64(16))):
+        got = oracle.words_to_normals(words).astype(np.float64)
+        ref = _libm_box_muller(words)
+        assert np.abs(got - ref).max() < 2e-6
+
+
 def test_normal_map_special_words():
     def word(k1, k2):
         return (k1 << 40) | (k2 << 16)
