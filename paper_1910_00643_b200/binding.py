@@ -72,8 +72,16 @@ def lib():
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: build it with "
-                              "`python -m paper_1910_00643_b200.build` (needs nvcc)")
+            # not built yet: compile it now (nvcc, sm_100a); one process at a time
+            import fcntl
+            from . import build as _build
+            try:
+                with open(os.path.join(_HERE, ".build.lock"), "w") as lock:
+                    fcntl.flock(lock, fcntl.LOCK_EX)
+                    if not os.path.exists(LIB_PATH):
+                        _build.build(force=True)
+            except Exception as exc:
+                raise ImportError(f"{LIB_PATH} is missing and could not be built with nvcc: {exc}") from exc
         L = C.CDLL(LIB_PATH)
         vp, u64, u32, i32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32
         sig = {
