@@ -1,7 +1,10 @@
 // K2, staged variant: the fused outer step of Algorithm 1 (exact average, Eq. 2, Eq. 3,
 // broadcast, buffer policy) with the replica rows moved by the bulk-copy engine (TMA).
 //
-// A persistent CTA owns column tiles of kTileCols columns. For each tile a producer thread
+// A persistent CTA (one per SM) owns column tiles of kTileCols = 4096 columns, i.e. 16 KB per row
+// segment: a bare bulk-copy pipeline measured 6.1 TB/s with 4 KB copies and 6.56 TB/s with 16 KB
+// ones (a plain vector copy: 6.8 TB/s), so the segments are made large and each consumer
+// thread handles kSub column groups of a tile. For each tile a producer thread
 // streams the m row segments (and, with the first of them, the anchor and u tiles) into a
 // ring of shared-memory stages with
 // cp.async.bulk (global -> shared, completion on an mbarrier); eight consumer warps add the
@@ -26,24 +29,32 @@
 
 namespace slowmo {
 
-constexpr int kTileCols = 1024;                    // columns per tile: 4 per consumer thread
+#ifndef SLOWMO_STAGED_TILE_COLS
+#define SLOWMO_STAGED_TILE_COLS 4096   // 16 KB per row segment: bulk copies of 4 KB top out near 6.1 TB/s
+#endif
+constexpr int kTileCols = SLOWMO_STAGED_TILE_COLS; // columns per tile
 #ifndef SLOWMO_STAGED_ROWS
-#define SLOWMO_STAGED_ROWS 4
+#define SLOWMO_STAGED_ROWS 2
 #endif
 #ifndef SLOWMO_STAGED_STAGES
-#define SLOWMO_STAGED_STAGES 4
+#define SLOWMO_STAGED_STAGES 2
 #endif
 #ifndef SLOWMO_STAGED_CTAS
-#define SLOWMO_STAGED_CTAS 2
+#define SLOWMO_STAGED_CTAS 1
 #endif
 constexpr int kStageRows = SLOWMO_STAGED_ROWS;     // row segments per pipeline stage
 constexpr int kStages = SLOWMO_STAGED_STAGES;      // ring depth
 #ifndef SLOWMO_STAGED_BULK_STORES
 #define SLOWMO_STAGED_BULK_STORES 1  // 1: rows written by bulk copies from shared memory; 0: by vector stores
 #endif
-constexpr int kOutBufs = 3;                        // output tiles in flight per CTA
+#ifndef SLOWMO_STAGED_OUT_BUFS
+#define SLOWMO_STAGED_OUT_BUFS 3
+#endif
+constexpr int kOutBufs = SLOWMO_STAGED_OUT_BUFS;                        // output tiles in flight per CTA
 constexpr int kConsumerWarps = 8;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kSub = kTileCols / (kConsumerThreads * 4);  // column groups per consumer thread and tile
+static_assert(kSub >= 1 && kSub * kConsumerThreads * 4 == kTileCols, "tile must be a multiple of 1024 columns");
 constexpr int kStagedThreads = kConsumerThreads + 64;  // + one load-producer warp + one store warp
 constexpr uint32_t kWaitTries = 1u << 20;          // bound of every mbarrier wait
 constexpr int kStagedCtasPerSm = SLOWMO_STAGED_CTAS;
@@ -177,38 +188,39 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
     }
   } else if (warp < kConsumerWarps) {
     // ---------------- consumers ----------------
+    // thread tid owns the column groups tid + k*kConsumerThreads (k < kSub) of the tile
     uint32_t job = 0, outs = 0;
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
       const uint32_t col0 = tile * kTileCols;
       const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
-      const bool active = tid * 4u < ncols;
-      const uint64_t col = (uint64_t)col0 + tid * 4u;
-
-      float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), u0 = x0;
+      float4 x0[kSub], u0[kSub];
 
       for (int pass = 0; pass < kPasses; ++pass) {
         // ordered sum over the workers, chunk by chunk
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 s[kSub];
         for (uint32_t c = 0; c < nchunks; ++c, ++job) {
           const uint32_t st = job % kStages, round = job / kStages;
           mbar_wait(&S.full[st], round & 1u, &S.abort, status, 2);
           const uint32_t rows = min((uint32_t)kStageRows, A.m - c * kStageRows);
-          if (active) {
+#pragma unroll
+          for (int k = 0; k < kSub; ++k) {
+            const uint32_t lc = (tid + k * kConsumerThreads) * 4u;  // column inside the tile
+            if (lc >= ncols) continue;
             if (pass == 0 && c == 0) {
-              x0 = *reinterpret_cast<const float4 *>(&S.stage[st][kAnchorSlot][tid * 4u]);
-              u0 = *reinterpret_cast<const float4 *>(&S.stage[st][kUSlot][tid * 4u]);
+              x0[k] = *reinterpret_cast<const float4 *>(&S.stage[st][kAnchorSlot][lc]);
+              u0[k] = *reinterpret_cast<const float4 *>(&S.stage[st][kUSlot][lc]);
             }
 #pragma unroll
             for (int r = 0; r < kStageRows; ++r) {
               if ((uint32_t)r < rows) {
-                const float4 v = *reinterpret_cast<const float4 *>(&S.stage[st][r][tid * 4u]);
+                const float4 v = *reinterpret_cast<const float4 *>(&S.stage[st][r][lc]);
                 if (c == 0 && r == 0) {
-                  s = v;
+                  s[k] = v;
                 } else {
-                  s.x = __fadd_rn(s.x, v.x);
-                  s.y = __fadd_rn(s.y, v.y);
-                  s.z = __fadd_rn(s.z, v.z);
-                  s.w = __fadd_rn(s.w, v.w);
+                  s[k].x = __fadd_rn(s[k].x, v.x);
+                  s[k].y = __fadd_rn(s[k].y, v.y);
+                  s[k].z = __fadd_rn(s[k].z, v.z);
+                  s[k].w = __fadd_rn(s[k].w, v.w);
                 }
               }
             }
@@ -216,44 +228,55 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
           __syncwarp();
           if ((tid & 31) == 0) mbar_arrive(&S.empty[st]);
         }
-        const float4 mean = make_float4(__fdiv_rn(s.x, A.m_float), __fdiv_rn(s.y, A.m_float),
-                                        __fdiv_rn(s.z, A.m_float), __fdiv_rn(s.w, A.m_float));
-        float4 outv = mean;  // passes 1, 2: averaged buffer
-        if (pass == 0) {
-          float4 un;
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            // Eq. (2) and Eq. (3)
-            const float ue = __fmaf_rn(A.beta, comp(u0, e), __fmul_rn(__fsub_rn(comp(x0, e), comp(mean, e)), A.inv_gamma));
-            comp(un, e) = ue;
-            comp(outv, e) = __fmaf_rn(A.neg_alpha_gamma, ue, comp(x0, e));
-          }
-          if (active && !S.abort) st_stream(A.u + col, un);
-        }
 
-#if !SLOWMO_STAGED_BULK_STORES
-        if (active && !S.abort) {
-          float *dst = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
-          store_rows(dst + col, A.pitch, A.m, outv);
-          if (pass == 0) {
-            st_stream(A.anchor + col, outv);
-            if (POLICY == 0) {
-              const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-              store_rows(A.h + col, A.pitch, A.m, zero);
-              if (NBUF == 2) store_rows(A.v + col, A.pitch, A.m, zero);
-            }
-          }
-        }
-        continue;
-#endif
         // the tile goes to shared memory once; the store warp sends it to every row
         const uint32_t ob = outs % kOutBufs, oround = outs / kOutBufs;
         ++outs;
+#if SLOWMO_STAGED_BULK_STORES
         mbar_wait(&S.out_empty[ob], (oround & 1u) ^ 1u, &S.abort, status, 3);
-        if (active) *reinterpret_cast<float4 *>(&S.out[ob][tid * 4u]) = outv;
+#endif
+#pragma unroll
+        for (int k = 0; k < kSub; ++k) {
+          const uint32_t lc = (tid + k * kConsumerThreads) * 4u;
+          if (lc >= ncols) continue;
+          const uint64_t col = (uint64_t)col0 + lc;
+          const float4 mean = make_float4(__fdiv_rn(s[k].x, A.m_float), __fdiv_rn(s[k].y, A.m_float),
+                                          __fdiv_rn(s[k].z, A.m_float), __fdiv_rn(s[k].w, A.m_float));
+          float4 outv = mean;  // passes 1, 2: averaged buffer
+          if (pass == 0) {
+            float4 un;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              // Eq. (2) and Eq. (3)
+              const float ue =
+                  __fmaf_rn(A.beta, comp(u0[k], e), __fmul_rn(__fsub_rn(comp(x0[k], e), comp(mean, e)), A.inv_gamma));
+              comp(un, e) = ue;
+              comp(outv, e) = __fmaf_rn(A.neg_alpha_gamma, ue, comp(x0[k], e));
+            }
+            if (!S.abort) st_stream(A.u + col, un);
+          }
+#if SLOWMO_STAGED_BULK_STORES
+          *reinterpret_cast<float4 *>(&S.out[ob][lc]) = outv;
+#else
+          if (!S.abort) {
+            float *dst = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
+            store_rows(dst + col, A.pitch, A.m, outv);
+            if (pass == 0) {
+              st_stream(A.anchor + col, outv);
+              if (POLICY == 0) {
+                const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+                store_rows(A.h + col, A.pitch, A.m, zero);
+                if (NBUF == 2) store_rows(A.v + col, A.pitch, A.m, zero);
+              }
+            }
+          }
+#endif
+        }
+#if SLOWMO_STAGED_BULK_STORES
         fence_async_proxy();
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(&S.out_full[ob]);
+#endif
       }
     }
   } else if (SLOWMO_STAGED_BULK_STORES && warp == kConsumerWarps + 1) {
