@@ -35,7 +35,9 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(_build.build())
+        import os
+        # tests that plant mistakes in a copy of the oracle point this at the copy's library
+        L = C.CDLL(os.environ.get("SLOWMO_ORACLE_LIB") or _build.build())
         L.oracle_mix64.restype = C.c_uint64
         L.oracle_mix64.argtypes = [C.c_uint64]
         L.oracle_stream_word.restype = C.c_uint64
