@@ -630,3 +630,50 @@ def test_full_size_staged_and_fused_outer_steps_equal_direct():
     for other in res[1:]:
         for a, b in zip(res[0], other):
             assert torch.equal(a[..., :w["P"]], b[..., :w["P"]])
+
+
+# ------------------------------------------------------------------ seeded random configurations
+
+def _random_case(rng):
+    base = rng.choice(["nesterov", "adam", "sgp_nesterov", "sgp_adam"])
+    no_average = bool(rng.random() < 0.25)
+    policy = rng.choice(["reset", "maintain"] if no_average else ["reset", "maintain", "average"])
+    supplied = bool(rng.random() < 0.3)
+    m = int(rng.choice([1, 2, 3, 5, 7, 8, 16, 33, 64]))
+    return dict(P=int(rng.integers(1, 6000)), m=m, tau=int(rng.integers(1, 6)), T=int(rng.integers(1, 4)),
+                alpha=float(rng.choice([1.0, 0.5, 1.5])), beta=float(rng.choice([0.0, 0.5, 0.9])),
+                gamma=float(rng.choice([1e-3, 0.01])) if "adam" in base else float(rng.choice([0.01, 0.1])),
+                base=str(base), mu=float(rng.choice([0.0, 0.9])), weight_decay=float(rng.choice([0.0, 1e-4, 1e-2])),
+                adam_b1=0.9, adam_b2=float(rng.choice([0.98, 0.999])), adam_eps=float(rng.choice([1e-8, 1e-6])),
+                buffer_policy=str(policy), grad_mode="supplied" if supplied else "generated",
+                seed=int(rng.integers(0, 2**40)), a_lo=0.1, a_hi=float(rng.choice([1.0, 3.0])),
+                c_std=float(rng.choice([0.05, 1.0])), sigma=float(rng.choice([0.0, 0.01, 0.3])),
+                x_init=float(rng.choice([0.0, -0.5])), no_average=no_average)
+
+
+@pytest.mark.parametrize("case", range(48))
+def test_seeded_random_configurations_match_the_oracle(case):
+    rng = np.random.Generator(np.random.PCG64(1000 + case))
+    w = _random_case(rng)
+    variant = str(rng.choice(["direct", "staged", "fused", "lazy"]))
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", variant)
+    grad = None
+    if w["grad_mode"] == "supplied":
+        grad = s.alloc_gradient()
+        s.fill_gradient()
+    gammas = None
+    if rng.random() < 0.3:   # a changing base learning rate
+        gammas = (w["gamma"] * rng.uniform(0.5, 2.0, size=w["T"])).astype(np.float32)
+    for t in range(w["T"]):
+        if gammas is not None:
+            s.set_gamma(float(gammas[t]))
+        left = w["tau"]
+        while left:          # the inner loop in random pieces
+            n = int(rng.integers(1, left + 1))
+            s.local_steps(n, grad)
+            left -= n
+        s.outer_step()
+    _check_against_oracle(s, w, np.arange(w["P"]), gamma_t=gammas, exact=True)
+    assert s.guards_intact(), (w, variant)
+    s.close()
