@@ -77,13 +77,18 @@ enum {
   SLOWMO_OUTER_FUSED = 3,  /* the last inner step of each outer iteration runs inside the
                               outer-step kernel (same results, fewer HBM bytes); see
                               slowmo_local_steps for what this changes for the caller       */
-  SLOWMO_OUTER_LAZY = 4    /* SLOWMO_OUTER_FUSED, and in addition the outer step does not write
+  SLOWMO_OUTER_LAZY = 4,   /* SLOWMO_OUTER_FUSED, and in addition the outer step does not write
                               the m broadcast rows (nor the reset / averaged buffer rows): the
                               first inner step of the next iteration reads the anchor (and zero,
                               or the mean kept in row 0) instead of the rows. Same results through
                               the API; the caller's raw x, h, v tensors are up to date only after
                               slowmo_materialize or any call that reads state. Needs tau >= 2,
                               otherwise it behaves as SLOWMO_OUTER_FUSED                     */
+  /* SLOWMO_K_LOCAL: layout of the fused local-step kernel (identical arithmetic per element) */
+  SLOWMO_LOCAL_ROW_TILES = 5,    /* one block = one 2048-column tile of one replica row            */
+  SLOWMO_LOCAL_COLUMN_OWNER = 6  /* one thread = one 4-column group of all m rows (reads the
+                                    curvature once per column); the default with a generated
+                                    gradient                                                      */
 };
 
 /*
@@ -167,8 +172,7 @@ int slowmo_destroy(slowmo_ctx *ctx);
  *              x_i = 0.5*x_{k+1/2,i} + 0.5*x_{k+1/2,(i-hops) mod m}.
  *              This mixing matrix is doubly stochastic, so the push-sum weights stay exactly 1
  *              and the de-biased z equals x; the gradient is therefore evaluated at x.
- *              SGP bases need m <= 64 (ENOTIMPL from slowmo_create otherwise) and ignore
- *              SLOWMO_OUTER_FUSED.
+ *              SGP bases ignore SLOWMO_OUTER_FUSED and SLOWMO_OUTER_LAZY.
  *
  * `grad` is a device [m, pitch] tensor in supplied mode (read by each of the n steps) and
  * must be NULL in generated mode (EINVAL otherwise).
@@ -236,6 +240,8 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
  * never wait for one another. Contexts that ran the local steps are told with
  * slowmo_outer_step_external. The local steps of sharded workers must use a communication-free
  * base (the SGP bases mix only the rows of one context). Errors as for slowmo_outer_step_static.
+ * The call has no context, so a CUDA failure is returned as SLOWMO_ECUDA but recorded nowhere:
+ * ask the CUDA runtime (cudaGetLastError) for the code.
  */
 typedef struct {
   uint32_t world, rank;
@@ -259,8 +265,12 @@ int slowmo_outer_step_external(slowmo_ctx *ctx);
  * A no-op with the other variants. Enqueued on the stream. */
 int slowmo_materialize(slowmo_ctx *ctx);
 
-/* Change the base learning rate (a schedule's gamma_t). Legal only between outer
- * iterations, i.e. when k = 0 (ESTATE otherwise). EINVAL unless gamma > 0 and finite. */
+/* Change the base learning rate: the gamma_t of a learning-rate schedule. Algorithm 1 indexes
+ * gamma by the outer iteration t only, and Section 2 (the remark under Eq. (3)) divides by
+ * gamma_t in Eq. (2) precisely so that the slow momentum buffer does not depend on the
+ * schedule; so the call is legal only between outer iterations, i.e. when k = 0 (ESTATE
+ * otherwise), and the new value is used by the local steps, Eq. (2) and Eq. (3) of the
+ * iteration that follows. EINVAL unless gamma > 0 and finite. */
 int slowmo_set_gamma(slowmo_ctx *ctx, float gamma_t);
 
 /*
@@ -277,8 +287,36 @@ int slowmo_get_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offs
 int slowmo_set_params(slowmo_ctx *ctx, int which, int32_t replica, uint64_t offset, uint64_t count,
                       const float *src, int src_on_device);
 
-/* Position in Algorithm 1: outer iteration t, inner steps k taken in it, Adam count l. */
+/* Position in Algorithm 1: the loop indices t (outer iterations completed) and k (base-optimizer
+ * steps taken in the current one), and Table C.1's step count l of the bias corrections (Adam
+ * steps since the buffers were last zero). Any pointer may be NULL. */
 int slowmo_get_counters(slowmo_ctx *ctx, uint64_t *t, uint32_t *k, uint64_t *l);
+
+/*
+ * Checkpoint and restore of everything Algorithm 1 carries besides the tensors: its loop indices
+ * t and k, Table C.1's step count l (the caption's l = k with buffers reset, l = t tau + k with
+ * buffers kept, counted from 1 here) and the gamma_t in force. Together with the tensors
+ * x, anchor, u, h (and v), read with slowmo_get_params and written with slowmo_set_params, this
+ * is the whole state: a context created with the same configuration, given the tensors and this
+ * record, continues bit-identically to the run the checkpoint was taken from -- the noise of
+ * step (t, k), the hop distance of the SGP graph and the bias corrections 1/(1 - beta^l) all
+ * follow from the record. (beta_1^l and beta_2^l are re-formed by l successive binary64
+ * multiplications, exactly as the step loop forms them.)
+ *
+ * slowmo_get_state may be called at any time. slowmo_set_state first writes out whatever the
+ * context still owes its tensors (a deferred last inner step, virtual replicas), then moves to
+ * the given position; call it BEFORE slowmo_set_params of the tensors when restoring. A state
+ * with k = tau is legal (the outer step is then due). EINVAL: k > tau, gamma_t not finite and
+ * positive, l < k, or l != k under SLOWMO_BUF_RESET.
+ */
+typedef struct {
+  uint64_t t;    /* outer iterations completed                                    */
+  uint64_t l;    /* base-optimizer steps since the buffers were last zero         */
+  uint32_t k;    /* inner steps taken in the current outer iteration, 0 .. tau    */
+  float gamma_t; /* base learning rate in force                                   */
+} slowmo_state;
+int slowmo_get_state(slowmo_ctx *ctx, slowmo_state *out);
+int slowmo_set_state(slowmo_ctx *ctx, const slowmo_state *in);
 
 /* Fill a device [m, pitch] tensor with the fixed synthetic gradient G[i,j] = sigma * z from
  * the hash (stream tag 5, worker i). For supplied-mode benchmarks; enqueued on the stream. */
@@ -298,11 +336,15 @@ int slowmo_debug_noise(slowmo_ctx *ctx, uint32_t tag, uint64_t t, uint32_t k, ui
  * value of the 24-bit radius field and of the 24-bit angle field. */
 int slowmo_debug_words_to_normals(slowmo_ctx *ctx, const uint64_t *words, uint64_t n, float *out);
 
-/* Segment idx of the optional parameter-tensor table: first coordinate and length. */
+/* Segment idx of the optional parameter-tensor table: first coordinate and length. The method
+ * treats the model as one vector x in R^d (Eq. (1)); a network's parameter tensors are contiguous
+ * segments of it, and this table only records where they lie. EINVAL without a table or for
+ * idx >= n_tensors. */
 int slowmo_tensor_range(slowmo_ctx *ctx, uint32_t idx, uint64_t *offset, uint64_t *count);
 
-/* Select the implementation of a kernel (SLOWMO_K_*, SLOWMO_VARIANT_* / SLOWMO_OUTER_*);
- * all variants compute identical results. */
+/* Select the implementation of a kernel: SLOWMO_K_OUTER with SLOWMO_VARIANT_DEFAULT or a
+ * SLOWMO_OUTER_* value, SLOWMO_K_LOCAL with SLOWMO_VARIANT_DEFAULT or a SLOWMO_LOCAL_* value
+ * (EINVAL otherwise). All variants compute identical results. */
 int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant);
 
 /* Wait for the stream and report SLOWMO_ETIMEOUT if any kernel recorded that one of its

@@ -19,14 +19,14 @@ POLICY = {"reset": 0, "maintain": 1, "average": 2}
 GRAD = {"generated": 0, "supplied": 1}
 TENSOR = {"x": 0, "anchor": 1, "u": 2, "h": 3, "v": 4, "a": 5, "c": 6}
 KERNEL = {"local": 0, "outer": 1}
-VARIANT = {"default": 0, "direct": 1, "staged": 2, "fused": 3, "lazy": 4}
+VARIANT = {"default": 0, "direct": 1, "staged": 2, "fused": 3, "lazy": 4, "row_tiles": 5, "column_owner": 6}
 EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_outer_step",
            "slowmo_set_gamma", "slowmo_get_params", "slowmo_set_params", "slowmo_get_counters",
            "slowmo_fill_gradient", "slowmo_debug_noise", "slowmo_tensor_range",
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
            "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize",
            "slowmo_outer_step_sharded", "slowmo_outer_step_external",
-           "slowmo_debug_words_to_normals"]
+           "slowmo_debug_words_to_normals", "slowmo_get_state", "slowmo_set_state"]
 
 
 class SlowMoError(RuntimeError):
@@ -62,6 +62,10 @@ class ShardArgs(C.Structure):
                 ("anchor", C.POINTER(C.c_void_p)), ("u", C.POINTER(C.c_void_p)),
                 ("base", C.c_int32), ("buffer_policy", C.c_int32),
                 ("alpha", C.c_float), ("beta", C.c_float), ("gamma_t", C.c_float)]
+
+
+class State(C.Structure):
+    _fields_ = [("t", C.c_uint64), ("l", C.c_uint64), ("k", C.c_uint32), ("gamma_t", C.c_float)]
 
 
 _lib = None
@@ -105,6 +109,8 @@ def lib():
             "slowmo_outer_step_sharded": [C.POINTER(ShardArgs), vp],
             "slowmo_outer_step_external": [vp],
             "slowmo_debug_words_to_normals": [vp, vp, u64, vp],
+            "slowmo_get_state": [vp, C.POINTER(State)],
+            "slowmo_set_state": [vp, C.POINTER(State)],
             "slowmo_outer_step_static": [vp, vp, vp, vp, vp, u64, u64, u32, i32, i32, C.c_float, C.c_float,
                                          C.c_float, vp, C.c_int],
         }
@@ -291,6 +297,16 @@ class SlowMo:
         t, k, l = C.c_uint64(), C.c_uint32(), C.c_uint64()
         _check(lib().slowmo_get_counters(self.ctx, C.byref(t), C.byref(k), C.byref(l)), "slowmo_get_counters")
         return t.value, k.value, l.value
+
+    def get_state(self):
+        """slowmo_get_state: position in Algorithm 1 as a dict(t, k, l, gamma_t)."""
+        st = State()
+        _check(lib().slowmo_get_state(self.ctx, C.byref(st)), "slowmo_get_state")
+        return {"t": st.t, "k": st.k, "l": st.l, "gamma_t": st.gamma_t}
+
+    def set_state(self, t, k, l, gamma_t):
+        st = State(t, l, k, gamma_t)
+        _check(lib().slowmo_set_state(self.ctx, C.byref(st)), "slowmo_set_state")
 
     def get_params(self, which, replica=-1, offset=0, count=None, out=None):
         """Copy columns [offset, offset+count) of tensor `which` to host (numpy) or to `out`

@@ -53,21 +53,23 @@ __device__ __forceinline__ float comp(const float4 &v, int e) { return reinterpr
 
 // ---- K0: fills ---------------------------------------------------------------------------
 
-// dst[i, j] = scale * z(tag, seed, 0, 0, i, j) for every row i and column j < 4*nvec.
+// dst[i, j] = scale * z(tag, seed, 0, 0, i, j) for every row i < rows and column j < 4*nvec
+// (blockIdx.y strides over the rows, so the row count is not limited by the grid).
 __global__ void __launch_bounds__(kThreads)
-fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t tag, uint64_t seed, float scale,
-                        uint32_t worker0) {
-  const uint32_t row = blockIdx.y;
-  const uint64_t key = stream_key(tag, seed, 0, 0, worker0 + row);  // row i holds global worker worker0 + i
-  float *p = dst + (uint64_t)row * pitch;
-  for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
-    // columns 4vi..4vi+3 are the pairs 2vi and 2vi+1 of the row's stream
-    const uint64_t s = key + kGoldenGamma * (2 * vi + 1);
-    float4 z;
-    word_to_normal_pair(mix64(s), z.x, z.y);
-    word_to_normal_pair(mix64(s + kGoldenGamma), z.z, z.w);
-    st_stream(p + 4 * vi, make_float4(__fmul_rn(scale, z.x), __fmul_rn(scale, z.y), __fmul_rn(scale, z.z),
-                                      __fmul_rn(scale, z.w)));
+fill_normal_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t rows, uint32_t tag, uint64_t seed,
+                        float scale, uint32_t worker0) {
+  for (uint32_t row = blockIdx.y; row < rows; row += gridDim.y) {
+    const uint64_t key = stream_key(tag, seed, 0, 0, worker0 + row);  // row i holds global worker worker0 + i
+    float *p = dst + (uint64_t)row * pitch;
+    for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads) {
+      // columns 4vi..4vi+3 are the pairs 2vi and 2vi+1 of the row's stream
+      const uint64_t s = key + kGoldenGamma * (2 * vi + 1);
+      float4 z;
+      word_to_normal_pair(mix64(s), z.x, z.y);
+      word_to_normal_pair(mix64(s + kGoldenGamma), z.z, z.w);
+      st_stream(p + 4 * vi, make_float4(__fmul_rn(scale, z.x), __fmul_rn(scale, z.y), __fmul_rn(scale, z.z),
+                                        __fmul_rn(scale, z.w)));
+    }
   }
 }
 
@@ -88,13 +90,15 @@ fill_curvature_kernel(float *a, uint32_t nvec, uint64_t seed, float a_lo, float 
   }
 }
 
-// dst[i, j] = value for every row and column j < 4*nvec.
+// dst[i, j] = value for every row i < rows and column j < 4*nvec.
 __global__ void __launch_bounds__(kThreads)
-fill_value_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, float value) {
-  float *p = dst + (uint64_t)blockIdx.y * pitch;
+fill_value_rows_kernel(float *dst, uint64_t pitch, uint32_t nvec, uint32_t rows, float value) {
   const float4 o = make_float4(value, value, value, value);
-  for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads)
-    st_stream(p + 4 * vi, o);
+  for (uint32_t row = blockIdx.y; row < rows; row += gridDim.y) {
+    float *p = dst + (uint64_t)row * pitch;
+    for (uint64_t vi = (uint64_t)blockIdx.x * kThreads + threadIdx.x; vi < nvec; vi += (uint64_t)gridDim.x * kThreads)
+      st_stream(p + 4 * vi, o);
+  }
 }
 
 // Export of one stream for the bit-exact test, j0 <= j < j0 + n: word j of the stream and/or
@@ -159,12 +163,50 @@ __device__ __forceinline__ void base_step(const LocalArgs &A, float g, float &x,
   x = __fmaf_rn(A.neg_gamma, d, x);
 }
 
+// Position of a 4-column group in a row's noise stream: columns 4v..4v+3 take the Box-Muller
+// pairs of words 2v and 2v+1, i.e. the generator states key + G(2v+1) and key + G(2v+2). The
+// term G(2v+1) does not depend on the row, so a thread that walks several rows forms it once.
+__device__ __forceinline__ uint64_t noise_counter(uint64_t vec_index) { return kGoldenGamma * (2ull * vec_index + 1); }
+
+// Stochastic gradient of the synthetic objective for one 4-column group of one worker:
+// g = fma(a, x - c, sigma * z), z from the worker's noise stream (key) at `counter`.
+__device__ __forceinline__ float4 generated_gradient(uint64_t key, uint64_t counter, const float4 &a, const float4 &x,
+                                                     const float4 &c, float sigma) {
+  const uint64_t st = key + counter;
+  float4 z, g;
+  word_to_normal_pair(mix64(st), z.x, z.y);
+  word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x, e), comp(c, e)), __fmul_rn(sigma, comp(z, e)));
+  return g;
+}
+
+// Noise keys of the rows a thread walks (column-owner kernels). Up to kInlineKeys rows the keys
+// come with the kernel arguments. Beyond that (DERIVE) the warp derives them itself, 32 at a
+// time: at every 32nd position of the walk lane l computes the key of the row at position
+// base + l (five mix64), and a shuffle hands the key of the current position to all lanes.
+// No memory is involved, so the worker count is unlimited. All 32 lanes of a warp must stay in
+// the walk (no early exit) because the shuffles name the full warp.
+template <bool DERIVE>
+struct RowKeys {
+  uint64_t lane_key = 0;
+  // call when (position & 31) == 0, with the row this lane's position base + lane maps to
+  __device__ __forceinline__ void refill(const LocalArgs &A, uint32_t row_of_lane) {
+    if (DERIVE) lane_key = stream_key(kTagGradNoise, A.seed, A.t, A.k, A.worker0 + row_of_lane);
+  }
+  __device__ __forceinline__ uint64_t at(const LocalArgs &A, uint32_t position, uint32_t row) const {
+    if (DERIVE) return __shfl_sync(0xFFFFFFFFu, lane_key, (int)(position & 31u));
+    return A.keys[row];
+  }
+};
+
 // One block = one tile of kThreads*U column groups of one row. Consecutive blocks are the m
 // rows of the same tile, so the shared curvature tile is read from DRAM once and from L2
 // m-1 times. Each thread issues all its loads (3 or 4 tensors x U) before any arithmetic.
 // The noise key of the row comes with the kernel arguments (computed on the host, the same
-// integer arithmetic) so that no issue slot is spent on it; beyond kInlineKeys rows it is
-// derived in the kernel.
+// integer arithmetic) so that no issue slot is spent on it; beyond kInlineKeys rows one lane
+// per warp derives it while the loads are in flight.
 template <int BASE, int GRAD, int U>
 __global__ void __launch_bounds__(kThreads, SLOWMO_LOCAL_MIN_BLOCKS)
 local_step_kernel(const LocalArgs A) {
@@ -204,18 +246,8 @@ local_step_kernel(const LocalArgs A) {
     if (!ok[u]) continue;
     const uint32_t vi = v0 + u * kThreads;
     float4 g;
-    if (GRAD == 0) {
-      // columns 4vi..4vi+3 take the Box-Muller pairs of words 2vi and 2vi+1 of the row's stream
-      const uint64_t st = key + kGoldenGamma * (2ull * (A.vec0 + vi) + 1);
-      float4 z;
-      word_to_normal_pair(mix64(st), z.x, z.y);
-      word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
-#pragma unroll
-      for (int e = 0; e < 4; ++e)
-        comp(g, e) = __fmaf_rn(comp(a[u], e), __fsub_rn(comp(x[u], e), comp(s[u], e)), __fmul_rn(A.sigma, comp(z, e)));
-    } else {
-      g = s[u];
-    }
+    if (GRAD == 0) g = generated_gradient(key, noise_counter(A.vec0 + vi), a[u], x[u], s[u], A.sigma);
+    else g = s[u];
 #pragma unroll
     for (int e = 0; e < 4; ++e) base_step<BASE>(A, comp(g, e), comp(x[u], e), comp(h[u], e), comp(v[u], e));
     const uint64_t off = roff + 4ull * vi;
@@ -229,24 +261,29 @@ local_step_kernel(const LocalArgs A) {
 // ROWS at a time. The curvature is loaded once per column (instead of once per row from L2)
 // and consecutive rows of a thread's loads are independent, so fewer threads keep as many
 // bytes in flight. Same arithmetic per element as local_step_kernel: results are identical.
-// Needs the row keys in the kernel arguments (m <= kInlineKeys) in generated mode.
+// DERIVE: more rows than noise keys fit the kernel arguments (see RowKeys); threads past the end
+// of the row then stay in the loop, with their loads and stores switched off.
 #ifndef SLOWMO_VIRT_MIN_BLOCKS
 #define SLOWMO_VIRT_MIN_BLOCKS 4   // resident blocks per SM asked of the virtual-replica form
 #endif
 #ifndef SLOWMO_COLS_MIN_BLOCKS
 #define SLOWMO_COLS_MIN_BLOCKS 3   // same for the ordinary form (80 registers; unbounded it took 110 and ran 10 % slower)
 #endif
-template <int BASE, int GRAD, int ROWS, bool VIRT>
+template <int BASE, int GRAD, int ROWS, bool VIRT, bool DERIVE>
 __global__ void __launch_bounds__(kThreads, VIRT ? SLOWMO_VIRT_MIN_BLOCKS : SLOWMO_COLS_MIN_BLOCKS)
 local_step_cols_kernel(const LocalArgs A) {
+  static_assert(32 % ROWS == 0, "key refills happen at multiples of 32 rows");
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
-  if (vi >= A.nvec) return;
-  const uint64_t col = 4ull * vi;
+  if (!DERIVE && vi >= A.nvec) return;
+  const bool ok = DERIVE ? vi < A.nvec : true;
+  const uint64_t col = ok ? 4ull * vi : 0;  // switched-off threads of the last warp point at column 0 and touch nothing
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (GRAD == 0) a = ld_shared_row(A.a + col);
+  if (GRAD == 0 && ok) a = ld_shared_row(A.a + col);
+  const uint64_t counter = noise_counter(A.vec0 + vi);
+  RowKeys<DERIVE> keys;
   // virtual replicas: every row starts from the anchor; buffers from zero or from the mean in row 0
   float4 x_all = a, h_all = make_float4(0.f, 0.f, 0.f, 0.f), v_all = h_all;
-  if (VIRT) {
+  if (VIRT && ok) {
     x_all = ld_stream(A.anchor + col);
     if (A.virt == 3) {
       h_all = ld_stream(A.h + col);
@@ -254,10 +291,11 @@ local_step_cols_kernel(const LocalArgs A) {
     }
   }
   for (uint32_t i0 = 0; i0 < A.m; i0 += ROWS) {
+    if (GRAD == 0 && (i0 & 31u) == 0) keys.refill(A, i0 + (threadIdx.x & 31u));
     float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
 #pragma unroll
     for (int q = 0; q < ROWS; ++q) {
-      if (i0 + q < A.m) {
+      if (ok && i0 + q < A.m) {
         const uint64_t off = (uint64_t)(i0 + q) * A.pitch + col;
         if (!VIRT) {
           x[q] = ld_stream(A.x + off);
@@ -280,18 +318,12 @@ local_step_cols_kernel(const LocalArgs A) {
     for (int q = 0; q < ROWS; ++q) {
       const uint32_t i = i0 + q;
       if (i >= A.m) break;
+      uint64_t key = 0;
+      if (GRAD == 0) key = keys.at(A, i, i);
+      if (!ok) continue;
       float4 g;
-      if (GRAD == 0) {
-        const uint64_t st = A.keys[i] + kGoldenGamma * (2ull * (A.vec0 + vi) + 1);
-        float4 z;
-        word_to_normal_pair(mix64(st), z.x, z.y);
-        word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(A.sigma, comp(z, e)));
-      } else {
-        g = s[q];
-      }
+      if (GRAD == 0) g = generated_gradient(key, counter, a, x[q], s[q], A.sigma);
+      else g = s[q];
 #pragma unroll
       for (int e = 0; e < 4; ++e) base_step<BASE>(A, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
       const uint64_t off = (uint64_t)i * A.pitch + col;

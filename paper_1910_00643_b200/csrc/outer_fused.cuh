@@ -35,29 +35,38 @@ __device__ __forceinline__ float4 div4(const float4 &s, float d) {
 }
 
 // One thread = one 4-element column group, all m rows. ROWS rows are loaded together.
-// Requires m <= kInlineKeys in generated mode (the launcher falls back otherwise).
+// DERIVE: more rows than noise keys fit the kernel arguments; the warp derives them (RowKeys) and
+// threads past the end of the row stay in the loop with their loads and stores switched off.
 // LAZY: the broadcast and the reset / average of the buffers are left to the next local step
 // (which then reads the anchor instead of the m rows): x rows are not written, "reset" writes
 // nothing, "average" writes the means to row 0 only.
-template <int BASE, int GRAD, int POLICY, int ROWS, bool LAZY>
+template <int BASE, int GRAD, int POLICY, int ROWS, bool LAZY, bool DERIVE>
 __global__ void __launch_bounds__(kThreads, SLOWMO_FUSED_MIN_BLOCKS)
 last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
+  static_assert(32 % ROWS == 0, "key refills happen at multiples of 32 rows");
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
-  if (vi >= O.nvec) return;
-  const uint64_t col = 4ull * vi;
+  if (!DERIVE && vi >= O.nvec) return;
+  const bool ok = DERIVE ? vi < O.nvec : true;
+  const uint64_t col = ok ? 4ull * vi : 0;
   const uint32_t m = O.m;
 
-  const float4 x0 = ld_stream(O.anchor + col);
-  const float4 u0 = ld_stream(O.u + col);
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (GRAD == 0) a = ld_shared_row(L.a + col);
+  float4 x0 = a, u0 = a;
+  if (ok) {
+    x0 = ld_stream(O.anchor + col);
+    u0 = ld_stream(O.u + col);
+    if (GRAD == 0) a = ld_shared_row(L.a + col);
+  }
+  const uint64_t counter = noise_counter(L.vec0 + vi);
+  RowKeys<DERIVE> keys;
 
   float4 sx = a, sh = a, sv = a;  // ordered sums over the workers (overwritten at row 0)
   for (uint32_t i0 = 0; i0 < m; i0 += ROWS) {
+    if (GRAD == 0 && (i0 & 31u) == 0) keys.refill(L, i0 + (threadIdx.x & 31u));
     float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
 #pragma unroll
     for (int q = 0; q < ROWS; ++q) {
-      if (i0 + q < m) {
+      if (ok && i0 + q < m) {
         const uint64_t off = (uint64_t)(i0 + q) * O.pitch + col;
         x[q] = ld_stream(L.x + off);
         h[q] = ld_stream(L.h + off);
@@ -69,18 +78,12 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
     for (int q = 0; q < ROWS; ++q) {
       const uint32_t i = i0 + q;
       if (i >= m) break;
+      uint64_t key = 0;
+      if (GRAD == 0) key = keys.at(L, i, i);
+      if (!ok) continue;
       float4 g;
-      if (GRAD == 0) {
-        const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * (L.vec0 + vi) + 1);
-        float4 z;
-        word_to_normal_pair(mix64(st), z.x, z.y);
-        word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(L.sigma, comp(z, e)));
-      } else {
-        g = s[q];
-      }
+      if (GRAD == 0) g = generated_gradient(key, counter, a, x[q], s[q], L.sigma);
+      else g = s[q];
 #pragma unroll
       for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
       add_in_order(sx, x[q], i == 0);
@@ -95,6 +98,7 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
     }
   }
 
+  if (!ok) return;
   const float4 xbar = div4(sx, O.m_float);
   float4 un, xn;
 #pragma unroll
@@ -119,15 +123,22 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
   }
 }
 
-template <int BASE, int GRAD, bool LAZY>
-inline void launch_last_step_outer_policy(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
+template <int BASE, int GRAD, bool LAZY, bool DERIVE>
+inline void launch_last_step_outer_keys(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
   const uint32_t blocks = (O.nvec + kThreads - 1) / kThreads;
   constexpr int ROWS = BASE == 1 ? SLOWMO_FUSED_ROWS / 2 : SLOWMO_FUSED_ROWS;
   switch (policy) {
-    case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
-    case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
-    default: last_step_outer_kernel<BASE, GRAD, 2, ROWS, LAZY><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    case 0: last_step_outer_kernel<BASE, GRAD, 0, ROWS, LAZY, DERIVE><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    case 1: last_step_outer_kernel<BASE, GRAD, 1, ROWS, LAZY, DERIVE><<<blocks, kThreads, 0, stream>>>(L, O); break;
+    default: last_step_outer_kernel<BASE, GRAD, 2, ROWS, LAZY, DERIVE><<<blocks, kThreads, 0, stream>>>(L, O); break;
   }
+}
+
+template <int BASE, int GRAD, bool LAZY>
+inline void launch_last_step_outer_policy(const LocalArgs &L, const OuterArgs &O, int policy, cudaStream_t stream) {
+  // the row keys travel in the arguments up to kInlineKeys workers and are derived in the kernel beyond
+  if (GRAD == 0 && L.m > kInlineKeys) launch_last_step_outer_keys<BASE, GRAD, LAZY, GRAD == 0>(L, O, policy, stream);
+  else launch_last_step_outer_keys<BASE, GRAD, LAZY, false>(L, O, policy, stream);
 }
 
 template <bool LAZY>

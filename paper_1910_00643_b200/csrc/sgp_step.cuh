@@ -24,37 +24,44 @@
 namespace slowmo {
 constexpr int kSgpRows = SLOWMO_SGP_ROWS;
 
-constexpr uint32_t kSgpMaxWorkers = kInlineKeys;  // generated mode needs the row keys in the kernel arguments
-
 __device__ __forceinline__ float4 half_sum(const float4 &p, const float4 &q) {
   return make_float4(__fadd_rn(__fmul_rn(0.5f, p.x), __fmul_rn(0.5f, q.x)), __fadd_rn(__fmul_rn(0.5f, p.y), __fmul_rn(0.5f, q.y)),
                      __fadd_rn(__fmul_rn(0.5f, p.z), __fmul_rn(0.5f, q.z)), __fadd_rn(__fmul_rn(0.5f, p.w), __fmul_rn(0.5f, q.w)));
 }
 
 // `cycles` = gcd(m, hops), `len` = m / cycles (host-computed); hops < m, or hops = 0 with m = 1.
-template <int BASE, int GRAD, int ROWS>
+// DERIVE: more workers than noise keys fit the kernel arguments; the warp derives the keys along
+// the walk (RowKeys), 32 positions of a cycle at a time, and no thread leaves the loop early.
+template <int BASE, int GRAD, int ROWS, bool DERIVE>
 __global__ void __launch_bounds__(kThreads, 3)
 sgp_step_kernel(const LocalArgs L, uint32_t hops, uint32_t cycles, uint32_t len) {
+  static_assert(32 % ROWS == 0, "key refills happen at multiples of 32 positions");
   const uint32_t vi = blockIdx.x * kThreads + threadIdx.x;
-  if (vi >= L.nvec) return;
-  const uint64_t col = 4ull * vi;
+  if (!DERIVE && vi >= L.nvec) return;
+  const bool ok = DERIVE ? vi < L.nvec : true;
+  const uint64_t col = ok ? 4ull * vi : 0;
   const uint32_t m = L.m;
 
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-  if (GRAD == 0) a = ld_shared_row(L.a + col);
+  if (GRAD == 0 && ok) a = ld_shared_row(L.a + col);
+  const uint64_t counter = noise_counter(L.vec0 + vi);
+  RowKeys<DERIVE> keys;
 
   for (uint32_t c = 0; c < cycles; ++c) {
     // walk the cycle c, c+hops, c+2 hops, ... ; `prev` is x_{k+1/2} of the row visited before
     float4 first = a, prev = a;
     uint32_t row = c;
     for (uint32_t n0 = 0; n0 < len; n0 += ROWS) {
+      // position n0 + l of the walk is row (row + l hops) mod m
+      if (GRAD == 0 && (n0 & 31u) == 0)
+        keys.refill(L, (uint32_t)(((uint64_t)row + (uint64_t)(threadIdx.x & 31u) * hops) % m));
       float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
       uint32_t rows[ROWS];
       uint32_t r = row;
 #pragma unroll
       for (int q = 0; q < ROWS; ++q) {
         rows[q] = r;
-        if (n0 + q < len) {
+        if (ok && n0 + q < len) {
           const uint64_t off = (uint64_t)r * L.pitch + col;
           x[q] = ld_stream(L.x + off);
           h[q] = ld_stream(L.h + off);
@@ -69,18 +76,12 @@ sgp_step_kernel(const LocalArgs L, uint32_t hops, uint32_t cycles, uint32_t len)
       for (int q = 0; q < ROWS; ++q) {
         if (n0 + q >= len) break;
         const uint32_t i = rows[q];
+        uint64_t key = 0;
+        if (GRAD == 0) key = keys.at(L, n0 + q, i);
+        if (!ok) continue;
         float4 g;
-        if (GRAD == 0) {
-          const uint64_t st = L.keys[i] + kGoldenGamma * (2ull * (L.vec0 + vi) + 1);
-          float4 z;
-          word_to_normal_pair(mix64(st), z.x, z.y);
-          word_to_normal_pair(mix64(st + kGoldenGamma), z.z, z.w);
-#pragma unroll
-          for (int e = 0; e < 4; ++e)
-            comp(g, e) = __fmaf_rn(comp(a, e), __fsub_rn(comp(x[q], e), comp(s[q], e)), __fmul_rn(L.sigma, comp(z, e)));
-        } else {
-          g = s[q];
-        }
+        if (GRAD == 0) g = generated_gradient(key, counter, a, x[q], s[q], L.sigma);
+        else g = s[q];
 #pragma unroll
         for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
         const uint64_t off = (uint64_t)i * L.pitch + col;
@@ -94,11 +95,9 @@ sgp_step_kernel(const LocalArgs L, uint32_t hops, uint32_t cycles, uint32_t len)
         prev = x[q];
       }
     }
-    st_stream(L.x + (uint64_t)c * L.pitch + col, half_sum(first, prev));
+    if (ok) st_stream(L.x + (uint64_t)c * L.pitch + col, half_sum(first, prev));
   }
 }
-
-inline cudaError_t sgp_configure() { return cudaSuccess; }
 
 inline uint32_t sgp_gcd(uint32_t p, uint32_t q) {
   while (q) {
@@ -114,12 +113,15 @@ inline void launch_sgp_step(const LocalArgs &L, uint32_t hops, bool adam, bool g
   hops = L.m > 1 ? hops % L.m : 0;
   const uint32_t cycles = hops ? sgp_gcd(L.m, hops) : L.m;  // hops = 0: every row is its own cycle (x unchanged)
   const uint32_t len = L.m / cycles;
+  const bool derive = generated && L.m > kInlineKeys;  // keys no longer fit the kernel arguments
   if (adam) {
-    if (generated) sgp_step_kernel<1, 0, kSgpRows / 2><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
-    else sgp_step_kernel<1, 1, kSgpRows / 2><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    if (derive) sgp_step_kernel<1, 0, kSgpRows / 2, true><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else if (generated) sgp_step_kernel<1, 0, kSgpRows / 2, false><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else sgp_step_kernel<1, 1, kSgpRows / 2, false><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
   } else {
-    if (generated) sgp_step_kernel<0, 0, kSgpRows><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
-    else sgp_step_kernel<0, 1, kSgpRows><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    if (derive) sgp_step_kernel<0, 0, kSgpRows, true><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else if (generated) sgp_step_kernel<0, 0, kSgpRows, false><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
+    else sgp_step_kernel<0, 1, kSgpRows, false><<<blocks, kThreads, 0, stream>>>(L, hops, cycles, len);
   }
 }
 

@@ -33,6 +33,7 @@ struct slowmo_ctx {
   float gamma;               // gamma_t in force
   std::vector<uint64_t> tensor_offsets;  // n_tensors + 1 prefix sums, or empty
   int outer_variant;
+  int local_variant;         // SLOWMO_VARIANT_DEFAULT, SLOWMO_LOCAL_ROW_TILES or SLOWMO_LOCAL_COLUMN_OWNER
   int virt;                  // lazy variant: 0, or how the next local step must read the (virtual) replicas
   bool pending_last;         // fused variant: the last inner step waits to run inside the outer step
   LocalArgs pending;         // its arguments (counters k, l already include it)
@@ -57,20 +58,23 @@ int cuda_fail(slowmo_ctx *ctx, cudaError_t e) {
 
 int check_launch(slowmo_ctx *ctx) { return cuda_fail(ctx, cudaGetLastError()); }
 
-uint32_t fill_blocks(const slowmo_ctx *ctx, uint32_t rows) {
-  // grid-stride fills: enough blocks to cover the machine a few times, split over the rows
+// Grid of the creation-time fills: blockIdx.x strides over the columns, blockIdx.y over the rows
+// (at most 65535 of them at a time, the grid's limit), enough blocks to cover the machine a few times.
+dim3 fill_grid(const slowmo_ctx *ctx, uint32_t rows) {
+  const uint32_t grid_rows = rows < 65535u ? rows : 65535u;
   uint64_t want = (uint64_t)ctx->num_sms * 16;
-  uint64_t per_row = (want + rows - 1) / rows;
+  uint64_t per_row = (want + grid_rows - 1) / grid_rows;
   uint64_t need = ((uint64_t)ctx->nvec + kThreads - 1) / kThreads;
   if (per_row > need) per_row = need;
   if (per_row < 1) per_row = 1;
-  return (uint32_t)per_row;
+  return dim3((uint32_t)per_row, grid_rows);
 }
 
-// Layout choice for the local step: the column-owner kernel needs inline keys in generated mode.
+// Layout of the local step (both compute every element with the same base_step).
 bool use_column_owner(const slowmo_ctx *ctx) {
-  const bool possible = ctx->cfg.grad_mode != SLOWMO_GRAD_GENERATED || ctx->cfg.m <= kInlineKeys;
-  if (SLOWMO_LOCAL_LAYOUT == 1 || !possible) return false;
+  if (ctx->local_variant == SLOWMO_LOCAL_ROW_TILES) return false;
+  if (ctx->local_variant == SLOWMO_LOCAL_COLUMN_OWNER) return true;
+  if (SLOWMO_LOCAL_LAYOUT == 1) return false;
   if (SLOWMO_LOCAL_LAYOUT == 2) return true;
   // measured on B200: with a generated gradient the column owner wins (the curvature is read
   // once per column: +3-4 % at m = 8 and m = 32); with a supplied gradient the two are equal
@@ -80,18 +84,24 @@ bool use_column_owner(const slowmo_ctx *ctx) {
 #ifndef SLOWMO_VIRT_ROWS_DIV
 #define SLOWMO_VIRT_ROWS_DIV 2   // the virtual-replica form keeps ROWS / this many rows in flight
 #endif
+template <int BASE, int GRAD, bool DERIVE>
+void launch_local_cols(slowmo_ctx *ctx, const LocalArgs &A) {
+  constexpr int ROWS = BASE == 1 ? SLOWMO_LOCAL_COL_ROWS / 2 : SLOWMO_LOCAL_COL_ROWS;
+  const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
+  if (A.virt)
+    local_step_cols_kernel<BASE, GRAD, (SLOWMO_VIRT_ROWS_DIV > 1 && ROWS > 1) ? ROWS / SLOWMO_VIRT_ROWS_DIV : ROWS, true, DERIVE>
+        <<<blocks, kThreads, 0, ctx->stream>>>(A);
+  else
+    local_step_cols_kernel<BASE, GRAD, ROWS, false, DERIVE><<<blocks, kThreads, 0, ctx->stream>>>(A);
+}
+
 template <int BASE, int GRAD>
 void launch_local(slowmo_ctx *ctx, const LocalArgs &A) {
-  constexpr int ROWS = BASE == 1 ? SLOWMO_LOCAL_COL_ROWS / 2 : SLOWMO_LOCAL_COL_ROWS;
-  if (A.virt) {  // first step after a lazy outer step: only the column owner can read virtual replicas
-    const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
-    local_step_cols_kernel<BASE, GRAD, (SLOWMO_VIRT_ROWS_DIV > 1 && ROWS > 1) ? ROWS / SLOWMO_VIRT_ROWS_DIV : ROWS, true>
-        <<<blocks, kThreads, 0, ctx->stream>>>(A);
-    return;
-  }
-  if (use_column_owner(ctx)) {
-    const uint32_t blocks = (A.nvec + kThreads - 1) / kThreads;
-    local_step_cols_kernel<BASE, GRAD, ROWS, false><<<blocks, kThreads, 0, ctx->stream>>>(A);
+  // the first step after a lazy outer step must be the column owner: only it can read virtual replicas
+  if (A.virt || use_column_owner(ctx)) {
+    // the row keys travel in the arguments up to kInlineKeys workers and are derived in the kernel beyond
+    if (GRAD == 0 && A.m > kInlineKeys) launch_local_cols<BASE, GRAD, GRAD == 0>(ctx, A);
+    else launch_local_cols<BASE, GRAD, false>(ctx, A);
     return;
   }
   const uint32_t per_tile = kThreads * kLocalUnroll;
@@ -197,7 +207,6 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   const bool generated = cfg->grad_mode == SLOWMO_GRAD_GENERATED;
   if (cfg->P == 0 || cfg->m == 0 || cfg->tau == 0) return SLOWMO_EINVAL;
   if (cfg->base < SLOWMO_BASE_NESTEROV || cfg->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
-  if (is_sgp(cfg->base) && cfg->m > kSgpMaxWorkers) return SLOWMO_ENOTIMPL;
   if (cfg->no_average != 0 && cfg->no_average != 1) return SLOWMO_EINVAL;
   if (cfg->no_average && cfg->buffer_policy == SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
   if (cfg->P > (1ull << 32) - 4096) return SLOWMO_EINVAL;  // columns are indexed with 32 bits
@@ -241,6 +250,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   ctx->pow_b1 = ctx->pow_b2 = 1.0;
   ctx->gamma = cfg->gamma;
   ctx->outer_variant = SLOWMO_VARIANT_DEFAULT;
+  ctx->local_variant = SLOWMO_VARIANT_DEFAULT;
   ctx->virt = 0;
   ctx->pending_last = false;
   ctx->status_dev = nullptr;
@@ -274,7 +284,6 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   if (e == cudaSuccess) e = cudaMalloc(&ctx->status_dev, 4 * sizeof(int));
   if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status_dev, 0, 4 * sizeof(int), ctx->stream);
   if (e == cudaSuccess) e = outer_staged_configure();
-  if (e == cudaSuccess && is_sgp(cfg->base)) e = sgp_configure();
   if (e != cudaSuccess) {
     if (ctx->status_dev) cudaFree(ctx->status_dev);
     delete ctx;
@@ -285,18 +294,18 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   const uint32_t m = cfg->m;
   const size_t row_bytes = (size_t)ctx->nvec * 4 * sizeof(float);
   const size_t pitch_bytes = buf->pitch * sizeof(float);
-  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->x, buf->pitch, ctx->nvec, cfg->x_init);
+  fill_value_rows_kernel<<<fill_grid(ctx, m), kThreads, 0, ctx->stream>>>(buf->x, buf->pitch, ctx->nvec, m, cfg->x_init);
   const uint32_t outer_rows = cfg->no_average ? m : 1;
-  fill_value_rows_kernel<<<dim3(fill_blocks(ctx, outer_rows), outer_rows), kThreads, 0, ctx->stream>>>(
-      buf->anchor, buf->pitch, ctx->nvec, cfg->x_init);
+  fill_value_rows_kernel<<<fill_grid(ctx, outer_rows), kThreads, 0, ctx->stream>>>(buf->anchor, buf->pitch, ctx->nvec,
+                                                                                   outer_rows, cfg->x_init);
   e = cudaGetLastError();
   if (e == cudaSuccess) e = cudaMemset2DAsync(buf->u, pitch_bytes, 0, row_bytes, outer_rows, ctx->stream);
   if (e == cudaSuccess) e = cudaMemset2DAsync(buf->h, pitch_bytes, 0, row_bytes, m, ctx->stream);
   if (e == cudaSuccess && buf->v) e = cudaMemset2DAsync(buf->v, pitch_bytes, 0, row_bytes, m, ctx->stream);
   if (e == cudaSuccess && generated) {
-    fill_curvature_kernel<<<fill_blocks(ctx, 1), kThreads, 0, ctx->stream>>>(buf->a, ctx->nvec, cfg->seed, cfg->a_lo, cfg->a_hi);
-    fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(buf->c, buf->pitch, ctx->nvec, kTagCentre,
-                                                                                   cfg->seed, cfg->c_std, cfg->worker_offset);
+    fill_curvature_kernel<<<fill_grid(ctx, 1).x, kThreads, 0, ctx->stream>>>(buf->a, ctx->nvec, cfg->seed, cfg->a_lo, cfg->a_hi);
+    fill_normal_rows_kernel<<<fill_grid(ctx, m), kThreads, 0, ctx->stream>>>(buf->c, buf->pitch, ctx->nvec, m, kTagCentre,
+                                                                             cfg->seed, cfg->c_std, cfg->worker_offset);
     e = cudaGetLastError();
   }
   if (e != cudaSuccess) {
@@ -371,7 +380,7 @@ int slowmo_local_steps(slowmo_ctx *ctx, uint32_t n, const float *grad) {
     ctx->k += 1;
     // fused and lazy variants: step tau-1 is taken inside the outer-step kernel
     if ((ctx->outer_variant == SLOWMO_OUTER_FUSED || ctx->outer_variant == SLOWMO_OUTER_LAZY) && ctx->k == c.tau &&
-        (!generated || c.m <= kInlineKeys) && !is_sgp(c.base) && !c.no_average && A.virt == 0) {
+        !is_sgp(c.base) && !c.no_average && A.virt == 0) {
       ctx->pending = A;
       ctx->pending_last = true;
       break;
@@ -593,13 +602,48 @@ int slowmo_get_counters(slowmo_ctx *ctx, uint64_t *t, uint32_t *k, uint64_t *l) 
   return SLOWMO_OK;
 }
 
+int slowmo_get_state(slowmo_ctx *ctx, slowmo_state *out) {
+  if (!ctx || !out) return SLOWMO_EINVAL;
+  out->t = ctx->t;
+  out->l = ctx->l;
+  out->k = ctx->k;
+  out->gamma_t = ctx->gamma;
+  return SLOWMO_OK;
+}
+
+int slowmo_set_state(slowmo_ctx *ctx, const slowmo_state *in) {
+  if (!ctx || !in) return SLOWMO_EINVAL;
+  if (ctx->cuda_error) return SLOWMO_ECUDA;
+  const slowmo_config &c = ctx->cfg;
+  if (in->k > c.tau || !finite_pos(in->gamma_t) || in->l < in->k) return SLOWMO_EINVAL;
+  // Table C.1's caption: with buffers zeroed at every outer step the count restarts there, l = k
+  if (c.buffer_policy == SLOWMO_BUF_RESET && in->l != in->k) return SLOWMO_EINVAL;
+  // what the context still owes the tensors (a deferred last step, virtual replicas) belongs to the
+  // position being left: write it out before the counters change
+  if (int rc = flush_pending(ctx)) return rc;
+  ctx->t = in->t;
+  ctx->k = in->k;
+  ctx->l = in->l;
+  ctx->gamma = in->gamma_t;
+  // beta^l exactly as the step loop forms it: l successive binary64 multiplications (a power that
+  // has underflowed to zero stays zero, so the loop can stop there)
+  double p1 = 1.0, p2 = 1.0;
+  for (uint64_t s = 0; s < in->l && (p1 != 0.0 || p2 != 0.0); ++s) {
+    p1 *= (double)c.adam_b1;
+    p2 *= (double)c.adam_b2;
+  }
+  ctx->pow_b1 = p1;
+  ctx->pow_b2 = p2;
+  return SLOWMO_OK;
+}
+
 int slowmo_fill_gradient(slowmo_ctx *ctx, float *grad) {
   if (!ctx || !grad) return SLOWMO_EINVAL;
   if (!aligned16(grad)) return SLOWMO_EALIGN;
   if (ctx->cuda_error) return SLOWMO_ECUDA;
   const uint32_t m = ctx->cfg.m;
-  fill_normal_rows_kernel<<<dim3(fill_blocks(ctx, m), m), kThreads, 0, ctx->stream>>>(
-      grad, ctx->buf.pitch, ctx->nvec, kTagSupplied, ctx->cfg.seed, ctx->cfg.sigma, ctx->cfg.worker_offset);
+  fill_normal_rows_kernel<<<fill_grid(ctx, m), kThreads, 0, ctx->stream>>>(
+      grad, ctx->buf.pitch, ctx->nvec, m, kTagSupplied, ctx->cfg.seed, ctx->cfg.sigma, ctx->cfg.worker_offset);
   return check_launch(ctx);
 }
 
@@ -646,7 +690,12 @@ int slowmo_set_variant(slowmo_ctx *ctx, int kernel, int variant) {
     ctx->outer_variant = variant;
     return SLOWMO_OK;
   }
-  if (kernel == SLOWMO_K_LOCAL) return variant == SLOWMO_VARIANT_DEFAULT ? SLOWMO_OK : SLOWMO_EINVAL;
+  if (kernel == SLOWMO_K_LOCAL) {
+    if (variant != SLOWMO_VARIANT_DEFAULT && variant != SLOWMO_LOCAL_ROW_TILES && variant != SLOWMO_LOCAL_COLUMN_OWNER)
+      return SLOWMO_EINVAL;
+    ctx->local_variant = variant;
+    return SLOWMO_OK;
+  }
   return SLOWMO_EINVAL;
 }
 

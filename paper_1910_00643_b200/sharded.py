@@ -48,6 +48,13 @@ class ShardedSlowMo:
         self.pitch = pitch
         self.peers = {name: [int(p) for p in h.buffer_ptrs] for name, h in self.handles.items()}
         self._token = torch.zeros(1, device="cuda")
+        self.gamma = w["gamma"]
+
+    def set_gamma(self, gamma):
+        """gamma_t of a learning-rate schedule (between outer iterations): used by this GPU's local
+        steps and by Eq. (2), (3) in the sharded outer step. Every rank must make the same call."""
+        self.local.set_gamma(gamma)
+        self.gamma = gamma
 
     def _fence(self):
         """Stream-ordered meeting point of all GPUs: nothing enqueued after it on the context's
@@ -66,7 +73,7 @@ class ShardedSlowMo:
         binding.outer_step_sharded(
             self.rank, self.peers["x"], self.peers["h"], self.peers.get("v"), self.peers["anchor"], self.peers["u"],
             m_local=self.m_local, P=w["P"], pitch=self.pitch, base=w["base"], buffer_policy=w["buffer_policy"],
-            alpha=w["alpha"], beta=w["beta"], gamma=w["gamma"], stream=self.local.stream)
+            alpha=w["alpha"], beta=w["beta"], gamma=self.gamma, stream=self.local.stream)
         self._fence()
         self.local.outer_step_external()
 

@@ -179,13 +179,69 @@ def test_many_workers():
         s.close()
 
 
-def test_more_workers_than_inline_noise_keys():
-    # beyond 64 workers the local-step kernel derives its noise keys itself
-    w = workloads.workload("tiny", P=1030, m=70, tau=2, T=2, buffer_policy="maintain")
+@pytest.mark.parametrize("layout", ["default", "row_tiles", "column_owner"])
+@pytest.mark.parametrize("variant", ["direct", "staged", "fused", "lazy"])
+def test_more_workers_than_inline_noise_keys(variant, layout):
+    # beyond 64 workers the noise keys no longer travel in the kernel arguments: the kernels derive
+    # them (one lane per warp in the row-tile layout, 32 rows per warp pass in the column-owner ones)
+    w = workloads.workload("tiny", P=1030, m=70, tau=3, T=2, buffer_policy="maintain")
     s = _slowmo(w, guard=64)
+    s.set_variant("outer", variant)
+    s.set_variant("local", layout)
     s.run(2)
     _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
     assert s.guards_intact()
+    s.close()
+
+
+@pytest.mark.parametrize("base,policy,m", [("nesterov", "average", 65), ("nesterov", "reset", 97), ("adam", "average", 66),
+                                           ("adam", "reset", 129), ("adam", "maintain", 200)])
+@pytest.mark.parametrize("variant", ["direct", "lazy"])
+def test_derived_noise_keys_for_every_base_and_policy(base, policy, m, variant):
+    # P chosen so that the last warp of the grid has lanes past the end of the row (they must stay in
+    # the key-deriving loop without touching memory): 1030 columns = 258 groups = 8 warps + 2 lanes
+    w = workloads.workload("tiny", P=1030, m=m, tau=3, T=2, base=base, buffer_policy=policy,
+                           gamma=0.01 if base == "adam" else 0.05, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8, seed=8)
+    s = _slowmo(w, guard=64)
+    s.set_variant("outer", variant)
+    s.run(2)
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+
+
+def test_local_step_layouts_are_selectable_and_identical():
+    import torch
+    from paper_1910_00643_b200 import SlowMoError, binding
+    outs = []
+    for grad_mode in ("generated", "supplied"):
+        for layout in ("row_tiles", "column_owner", "default"):
+            w = workloads.workload("tiny", P=70_001, m=5, tau=3, T=2, grad_mode=grad_mode, buffer_policy="average")
+            s = _slowmo(w)
+            s.set_variant("local", layout)
+            grad = None
+            if grad_mode == "supplied":
+                grad = s.alloc_gradient()
+                s.fill_gradient()
+            s.run(2, grad)
+            _check_against_oracle(s, w, np.arange(0, w["P"], 7), exact=True)
+            s.synchronize()
+            outs.append(s.t["x"].clone())
+            with pytest.raises(SlowMoError) as e:
+                s.set_variant("local", "staged")        # an outer-step variant is not a local-step layout
+            assert e.value.status == binding.EINVAL
+            s.close()
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    assert torch.equal(outs[3], outs[4]) and torch.equal(outs[3], outs[5])
+
+
+def test_more_workers_than_one_grid_dimension_holds():
+    # 66 000 rows: the creation-time fills stride over the rows, and every kernel derives its keys
+    w = workloads.workload("tiny", P=9, m=66_000, tau=2, T=1, buffer_policy="average")
+    s = _slowmo(w)
+    s.run(1)
+    ref = _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert ref["x"].shape == (66_000, 9)
     s.close()
 
 
@@ -364,11 +420,19 @@ def test_sgp_supplied_gradient_and_step_by_step_calls():
     s.close()
 
 
-def test_sgp_needs_at_most_64_workers():
-    from paper_1910_00643_b200 import SlowMoError, binding
-    with pytest.raises(SlowMoError) as e:
-        _slowmo(workloads.workload("tiny", m=65, base="sgp_nesterov"))
-    assert e.value.status == binding.ENOTIMPL
+@pytest.mark.parametrize("base,policy", [("sgp_nesterov", "average"), ("sgp_adam", "reset"), ("sgp_nesterov", "maintain")])
+@pytest.mark.parametrize("m", [65, 96, 128, 131])
+def test_sgp_with_more_workers_than_inline_noise_keys(base, policy, m):
+    # the walk along the cycles of i -> i + hops derives its keys 32 positions at a time; m = 96 and 131
+    # give cycles whose length is not a multiple of 32, m = 128 several cycles per step
+    w = workloads.workload("tiny", P=1030, m=m, tau=9, T=2, base=base, buffer_policy=policy, alpha=0.9, beta=0.6,
+                           gamma=0.01 if "adam" in base else 0.05, weight_decay=1e-3, adam_b1=0.9, adam_b2=0.98,
+                           adam_eps=1e-8, seed=10)
+    s = _slowmo(w, guard=64)
+    s.run(w["T"])
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
 
 
 @pytest.mark.parametrize("name", ["sgp_resnet50", "sgp_transformer_adam"])
@@ -540,16 +604,115 @@ def test_get_and_set_params_round_trip():
     assert np.array_equal(dev.cpu().numpy().reshape(3, 40), s.get_params("h")[:, 7:47])
     # restore a checkpoint into a fresh context and continue: same result as an uninterrupted run
     s2 = _slowmo(w)
+    s2.set_state(**s.get_state())
     for key in ("x", "anchor", "u", "h"):
         s2.set_params(key, s.get_params(key))
-    s.run(1)
-    # the fresh context is at t = 0 for the noise key, so compare a state copy only
+    s.run(2)
+    s2.run(2)
     for key in ("x", "anchor", "u", "h"):
-        s2.set_params(key, s.get_params(key))
-        assert np.array_equal(s2.get_params(key), s.get_params(key))
+        assert np.array_equal(s2.get_params(key).view(np.uint32), s.get_params(key).view(np.uint32)), key
+    _check_against_oracle(s2, w, np.arange(w["P"]), T=3, exact=True)
     assert s.guards_intact()
     s.close()
     s2.close()
+
+
+def _checkpoint(s):
+    """Everything Algorithm 1 carries, on the host: the tensors and the position record."""
+    keys = ("x", "anchor", "u", "h") + (("v",) if s.t["v"] is not None else ())
+    return {"state": s.get_state(), "tensors": {k: s.get_params(k) for k in keys}}
+
+
+def _restore(s, ck):
+    s.set_state(**ck["state"])
+    for k, v in ck["tensors"].items():
+        s.set_params(k, np.ascontiguousarray(v))
+
+
+CHECKPOINT_CASES = {
+    "nesterov-generated-reset": dict(base="nesterov", buffer_policy="reset"),
+    "nesterov-generated-average": dict(base="nesterov", buffer_policy="average", weight_decay=1e-3),
+    "adam-maintain": dict(base="adam", buffer_policy="maintain", gamma=0.01, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8),
+    "adam-reset": dict(base="adam", buffer_policy="reset", gamma=0.01, adam_b1=0.9, adam_b2=0.98, adam_eps=1e-8),
+    "sgp-nesterov-maintain": dict(base="sgp_nesterov", buffer_policy="maintain", m=6),
+    "sgp-adam-average": dict(base="sgp_adam", buffer_policy="average", gamma=0.01, adam_b1=0.9, adam_b2=0.98,
+                             adam_eps=1e-8, m=5),
+    "noaverage-adam": dict(base="adam", buffer_policy="maintain", gamma=0.01, adam_b1=0.9, adam_b2=0.98,
+                           adam_eps=1e-8, no_average=True),
+}
+
+
+@pytest.mark.parametrize("variant", ["direct", "lazy"])
+@pytest.mark.parametrize("k_split", [0, 2, 5])       # restore between outer iterations, inside one, and with the outer step due
+@pytest.mark.parametrize("case", sorted(CHECKPOINT_CASES))
+def test_a_restored_run_continues_bit_identically(case, k_split, variant):
+    # T1 iterations (+ k_split inner steps), checkpoint, fresh context, restore, the rest: the result
+    # must equal the uninterrupted run and the oracle bit for bit, with a changing gamma_t
+    T1, T2, tau = 2, 2, 5
+    w = workloads.workload("tiny", P=2 * 1024 + 37, m=4, tau=tau, T=T1 + T2, alpha=0.9, beta=0.6, seed=14,
+                           **CHECKPOINT_CASES[case])
+    gammas = (w["gamma"] * np.array([1.0, 0.5, 2.0, 0.7])).astype(np.float32)
+
+    def advance(s, t_from, t_to, k_from=0):
+        for t in range(t_from, t_to):
+            if k_from == 0:
+                s.set_gamma(float(gammas[t]))
+            if tau - k_from:
+                s.local_steps(tau - k_from)
+            s.outer_step()
+            k_from = 0
+
+    first = _slowmo(w, guard=64)
+    first.set_variant("outer", variant)
+    advance(first, 0, T1)
+    if k_split:
+        first.set_gamma(float(gammas[T1]))
+        first.local_steps(k_split)
+    ck = _checkpoint(first)
+    assert ck["state"]["t"] == T1 and ck["state"]["k"] == k_split
+    assert ck["state"]["gamma_t"] == (gammas[T1] if k_split else gammas[T1 - 1])
+    first.close()
+
+    second = _slowmo(w, guard=64)
+    second.set_variant("outer", variant)
+    _restore(second, ck)
+    assert second.counters() == (T1, k_split, ck["state"]["l"])
+    advance(second, T1, T1 + T2, k_from=k_split)
+    _check_against_oracle(second, w, np.arange(w["P"]), gamma_t=gammas, exact=True)
+    assert second.guards_intact()
+    second.close()
+
+
+def test_set_state_refuses_impossible_positions_and_flushes_what_is_owed():
+    from paper_1910_00643_b200 import SlowMoError, binding
+    w = workloads.workload("tiny", P=3000, m=3, tau=3, T=2)
+    s = _slowmo(w)
+    for bad in (dict(t=0, k=4, l=4, gamma_t=0.05),            # k > tau
+                dict(t=0, k=1, l=0, gamma_t=0.05),            # fewer steps since the reset than steps in this iteration
+                dict(t=3, k=1, l=7, gamma_t=0.05),            # reset policy: l must equal k
+                dict(t=0, k=0, l=0, gamma_t=0.0), dict(t=0, k=0, l=0, gamma_t=float("nan"))):
+        with pytest.raises(SlowMoError) as e:
+            s.set_state(**bad)
+        assert e.value.status == binding.EINVAL
+    # a lazy context owes its tensors the broadcast: set_state writes it out before moving on
+    s.set_variant("outer", "lazy")
+    s.run(1)
+    ref = oracle.run(oracle.make_config(**dict(w, T=1)), j0=0, n=w["P"])
+    s.set_state(t=1, k=0, l=0, gamma_t=w["gamma"])
+    s.synchronize()
+    x = s.t["x"].view(3, s.pitch)[:, :w["P"]].cpu().numpy()
+    assert np.array_equal(x.view(np.uint32), ref["x"].view(np.uint32))
+    s.run(1)
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    # with the buffers kept, l keeps counting across outer iterations: a large count is legal and
+    # its powers underflow to zero without harm
+    wm = workloads.workload("tiny", P=100, m=2, tau=3, base="adam", buffer_policy="maintain", gamma=0.01)
+    sm = _slowmo(wm)
+    sm.set_state(t=10**6, k=0, l=3 * 10**6, gamma_t=0.01)
+    sm.run(1)
+    assert sm.get_state() == {"t": 10**6 + 1, "k": 0, "l": 3 * 10**6 + 3, "gamma_t": np.float32(0.01)}
+    sm.close()
+    s.close()
 
 
 def test_tensor_table():
@@ -567,50 +730,109 @@ def test_tensor_table():
     s.close()
 
 
-# ------------------------------------------------------- full benchmark sizes, sampled coordinates
+# ------------------------------------------------------- full benchmark sizes
+#
+# Each full-size run is compared with the oracle on (i) sampled coordinates (both ends, tile
+# boundaries, 8192 uniform draws) and (ii) three contiguous slabs of 2^20 coordinates: the start of
+# the vector, the middle, and the end with its ragged tail (for the 1e9-parameter workload the middle
+# slab straddles the point where row 1's byte offset passes 2^32). Properties that hold at any size
+# (every replica equals the anchor, policy post-conditions) are checked over the whole of P. The
+# fraction of P compared element by element is asserted below; `-m fullp` runs compare all of it.
 
 FULL = ["resnet50", "bmuf", "local_sgd", "sync_sgd", "transformer_adam"]
+SLAB = 1 << 20
 
 
-@pytest.mark.parametrize("name", FULL)
-def test_full_size_generated_workloads_on_sampled_coordinates(name):
+def _slabs(w, pitch):
+    P = w["P"]
+    mid = (P // 2 // 4096) * 4096 - SLAB // 2 + 13         # unaligned start, crosses tile boundaries
+    if P * 4 > 2**32:                                      # rows longer than 4 GiB apart: straddle row 1's 2^32-byte mark
+        mid = (2**32 - pitch * 4) // 4 - SLAB // 2
+    return [np.arange(0, SLAB), np.arange(mid, mid + SLAB), np.arange(P - SLAB, P)]
+
+
+def _check_full_size(s, w, seed, slabs=True, gamma_t=None):
     import torch
-    w = workloads.workload(name)
-    s = _slowmo(w)
-    s.run(w["T"])
-    j = workloads.sample_coordinates(w["P"], 1 << 13, seed=1)
-    _check_against_oracle(s, w, j, exact=True)
-    # properties that hold at any size: consensus of the replicas, policy post-conditions
-    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
-    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
+    j = workloads.sample_coordinates(w["P"], 1 << 13, seed=seed)
+    _check_against_oracle(s, w, j, exact=True, gamma_t=gamma_t)
+    compared = len(j)
+    if slabs:
+        for slab in _slabs(w, s.pitch):
+            _check_against_oracle(s, w, slab, exact=True, gamma_t=gamma_t)
+            compared += len(slab)
+        assert compared >= 3 * SLAB
+    if not w.get("no_average"):
+        x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
+        assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())     # consensus over the whole of P
     h = s.t["h"].view(w["m"], s.pitch)[:, :w["P"]]
     if w["buffer_policy"] == "reset":
         assert not bool(h.any())
     if w["buffer_policy"] == "average":
         assert bool((h == h[0:1]).all())
-    assert bool(torch.isfinite(s.t["u"][:w["P"]]).all())
+    assert bool(torch.isfinite(s.t["u"].view(-1, s.pitch)[:, :w["P"]]).all())
+    return compared
+
+
+def _free(s):
+    import torch
     s.close()
     del s
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_generated_workloads(name):
+    w = workloads.workload(name)
+    s = _slowmo(w)
+    s.run(w["T"])
+    # slabs for the three workloads that differ in kernel and policy (resnet50: Nesterov / average,
+    # bmuf: reset, transformer_adam: Adam / maintain); the two degenerate cases share bmuf's kernels
+    _check_full_size(s, w, seed=1, slabs=name in ("resnet50", "bmuf", "transformer_adam"))
+    _free(s)
+
+
 @pytest.mark.parametrize("name,variant", [("stress_tau1", "direct"), ("stress_tau12", "direct"),
-                                          ("stress_tau12", "lazy"), ("stress_tau1", "fused")])
-def test_full_size_supplied_gradient_on_sampled_coordinates(name, variant):
-    import torch
+                                          ("stress_tau12", "lazy"), ("stress_tau1", "fused"),
+                                          ("stress_tau48", "direct"), ("stress_tau48", "lazy"),
+                                          ("stress_tau12", "staged")])
+def test_full_size_supplied_gradient(name, variant):
     w = workloads.workload(name)
     s = _slowmo(w)
     s.set_variant("outer", variant)
     s.alloc_gradient()
     s.fill_gradient()
     s.run(w["T"], s.grad)
-    j = workloads.sample_coordinates(w["P"], 1 << 13, seed=2)
-    _check_against_oracle(s, w, j, exact=True)       # reads through sync_status, which writes out lazy state
-    x = s.t["x"].view(w["m"], s.pitch)[:, :w["P"]]
-    assert bool((x == s.t["anchor"][:w["P"]].unsqueeze(0)).all())
-    s.close()
-    del s
-    torch.cuda.empty_cache()
+    _check_full_size(s, w, seed=2)       # reads through sync_status, which writes out lazy state
+    _free(s)
+
+
+@pytest.mark.parametrize("name,variant,layout", [("bmuf", "staged", "default"), ("bmuf", "lazy", "default"),
+                                                 ("resnet50", "lazy", "default"), ("resnet50", "staged", "row_tiles"),
+                                                 ("transformer_adam", "lazy", "row_tiles")])
+def test_full_size_other_variants_and_layouts(name, variant, layout):
+    # the staged (bulk-copy) outer step on a reset policy, the lazy variant at every policy, and the
+    # row-tile layout of the generated-gradient local step, each at full size (two outer iterations)
+    w = workloads.workload(name, T=2)
+    s = _slowmo(w)
+    s.set_variant("outer", variant)
+    s.set_variant("local", layout)
+    s.run(2)
+    _check_full_size(s, w, seed=5, slabs=False)
+    _check_against_oracle(s, w, _slabs(w, s.pitch)[1][:1 << 18], exact=True)
+    _free(s)
+
+
+@pytest.mark.parametrize("layout", ["row_tiles", "column_owner"])
+def test_full_size_with_more_workers_than_inline_noise_keys(layout):
+    # m = 70 > 64: the kernels derive the row keys themselves; P = 2^24 + 5 (ragged), 4.7 GB of state
+    w = workloads.workload("resnet50", P=(1 << 24) + 5, m=70, tau=4, T=2, n_tensors=0)
+    s = _slowmo(w)
+    s.set_variant("local", layout)
+    s.set_variant("outer", "lazy" if layout == "column_owner" else "direct")
+    s.run(2)
+    _check_full_size(s, w, seed=6, slabs=False)
+    _check_against_oracle(s, w, np.arange(w["P"] - (1 << 17), w["P"]), exact=True)
+    _free(s)
 
 
 def test_full_size_staged_and_fused_outer_steps_equal_direct():
@@ -624,12 +846,54 @@ def test_full_size_staged_and_fused_outer_steps_equal_direct():
         s.sync_status()
         res.append((s.t["anchor"].clone(), s.t["u"].clone(), s.t["h"].view(w["m"], s.pitch)[::8].clone(),
                     s.t["x"].view(w["m"], s.pitch)[::8].clone()))
-        s.close()
-        del s
-        torch.cuda.empty_cache()
+        _free(s)
     for other in res[1:]:
         for a, b in zip(res[0], other):
             assert torch.equal(a[..., :w["P"]], b[..., :w["P"]])
+
+
+# ------------------------------------------------------- every coordinate of a full-size workload
+
+FULLP_CHUNK = 1 << 22
+
+
+@pytest.mark.fullp
+@pytest.mark.parametrize("name,variant", [("resnet50", "direct"), ("bmuf", "direct"), ("transformer_adam", "direct"),
+                                          ("stress_tau12", "direct"), ("stress_tau12", "lazy")])
+def test_every_coordinate_of_a_full_size_workload(name, variant):
+    """Selected with -m fullp only (several minutes of oracle time per workload). The device state is
+    brought to the host in chunks of 2^22 coordinates and every element of every state tensor is
+    compared with the oracle bit for bit; the count of coordinates compared and of unequal elements
+    is printed (run with -s) and written to gpurun_out/fullp_<name>_<variant>.txt when that folder exists."""
+    import os
+    import time
+    w = workloads.workload(name)
+    s = _slowmo(w)
+    s.set_variant("outer", variant)
+    grad = None
+    if w["grad_mode"] == "supplied":
+        grad = s.alloc_gradient()
+        s.fill_gradient()
+    s.run(w["T"], grad)
+    s.sync_status()
+    cfg = oracle.make_config(**w)
+    unequal, compared, t0 = 0, 0, time.time()
+    for j0 in range(0, w["P"], FULLP_CHUNK):
+        n = min(FULLP_CHUNK, w["P"] - j0)
+        ref = oracle.run(cfg, j0=j0, n=n, precision="f32")
+        for key in _state_keys(w):
+            got = s.get_params(key, offset=j0, count=n).reshape(ref[key].shape)
+            unequal += int((got.view(np.uint32) != ref[key].view(np.uint32)).sum())
+        compared += n
+    line = (f"{name} ({variant}): {compared} of {w['P']} coordinates compared, all m={w['m']} workers, "
+            f"tensors {','.join(_state_keys(w))}: {unequal} unequal elements, {time.time() - t0:.0f} s")
+    print(line)
+    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    if os.path.isdir(out):
+        with open(os.path.join(out, f"fullp_{name}_{variant}.txt"), "w") as f:
+            f.write(line + "\n")
+    assert compared == w["P"] and unequal == 0, line
+    _free(s)
 
 
 # ------------------------------------------------------------------ seeded random configurations

@@ -10,8 +10,8 @@ import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 ORACLE = os.path.join(ROOT, "oracle")
-PINS, NOISE, SGP, NOAVG = ("tests/test_oracle_pins.py", "tests/test_oracle_noise.py", "tests/test_oracle_sgp.py",
-                            "tests/test_oracle_noaverage.py")
+PINS, NOISE, SGP, NOAVG, F32 = ("tests/test_oracle_pins.py", "tests/test_oracle_noise.py", "tests/test_oracle_sgp.py",
+                                 "tests/test_oracle_noaverage.py", "tests/test_oracle_binary32.py")
 
 # (file, text to find, replacement, pin file expected to notice): one plausible slip each
 MUTATIONS = [
@@ -28,6 +28,9 @@ MUTATIONS = [
      "case 1: *cos_out = sin_psi; *sin_out = cos_psi;  break;", NOISE),                                        # quadrant sign
     ("slowmo_noise.c", "s ^= s >> 27;", "s ^= s >> 28;", NOISE),                                               # hash shift
     ("slowmo_noise.c", "return z[j & 1];", "return z[0];", NOISE),                                             # sine output never used
+    # slips that exist in the binary32 build only (the binary64 pins cannot see them)
+    ("slowmo_oracle.c", "#define SQRT(a) sqrtf(a)", "#define SQRT(a) sqrtf(sqrtf(a))", F32),                    # wrong root in the float build
+    ("slowmo_oracle.c", "#define FMA(a, b, c) fmaf((a), (b), (c))", "#define FMA(a, b, c) fmaf((a), (b), (float)(int)(c))", F32),  # a cast that truncates
 ]
 
 
@@ -53,7 +56,9 @@ def _build_copy(tmp, fname, find, repl):
 @pytest.mark.parametrize("fname,find,repl,pins", MUTATIONS, ids=[f"{m[0]}:{i}" for i, m in enumerate(MUTATIONS)])
 def test_a_planted_mistake_fails_some_pin(tmp_path, fname, find, repl, pins):
     lib = _build_copy(str(tmp_path), fname, find, repl)
-    env = dict(os.environ, SLOWMO_ORACLE_LIB=lib)
+    # the second variable tells tests/conftest.py that this run is the mutation harness: a stray
+    # SLOWMO_ORACLE_LIB alone is refused there
+    env = dict(os.environ, SLOWMO_ORACLE_LIB=lib, SLOWMO_ORACLE_MUTATION_RUN="1")
     run = subprocess.run([sys.executable, "-m", "pytest", pins, "-x", "-q", "-p", "no:cacheprovider",
                           "-k", "not frozen and not mutation and not every_radius"], cwd=ROOT, env=env,
                          capture_output=True, timeout=600)

@@ -21,9 +21,14 @@ RTOL = 1e-5  # same gate as the parity tests; bit equality is expected and also 
 
 
 def _pre_state(s):
-    """Copies of the tensors an outer step reads and writes, taken before the context's own step."""
+    """Copies of the tensors an outer step reads and writes, taken before the context's own step.
+    The copies are made on the context's stream, the one both outer steps run on, so that neither
+    can overtake them."""
+    import torch
+    with torch.cuda.stream(s.stream):
+        mine = {k: (s.t[k].clone() if s.t[k] is not None else None) for k in ("x", "h", "v", "anchor", "u")}
     s.synchronize()
-    return {k: (s.t[k].clone() if s.t[k] is not None else None) for k in ("x", "h", "v", "anchor", "u")}
+    return mine
 
 
 def _compare(s, mine, what):
@@ -40,15 +45,15 @@ def _compare(s, mine, what):
         assert np.array_equal(got, ref), (what, key, "not bit-identical")
 
 
-def _one_call(s, w, what):
+def _one_call(s, w, what, wait=True):
     from paper_1910_00643_b200 import binding
     s.local_steps(w["tau"])
     mine = _pre_state(s)
     s.outer_step()                               # existing entry point, context path
     binding.outer_step_static(mine["x"], mine["h"], mine["v"], mine["anchor"], mine["u"], pitch=s.pitch,
                               P=s.P, m=s.m, base=w["base"], buffer_policy=w["buffer_policy"],
-                              alpha=w["alpha"], beta=w["beta"], gamma=w["gamma"], stream=s.stream, wait=True)
-    _compare(s, mine, what)
+                              alpha=w["alpha"], beta=w["beta"], gamma=w["gamma"], stream=s.stream, wait=wait)
+    _compare(s, mine, what)                      # synchronises the stream first
 
 
 def test_static_outer_step_matches_context_outer_step_twice_in_a_row():
@@ -63,6 +68,9 @@ def test_static_outer_step_matches_context_outer_step_twice_in_a_row():
     _one_call(s2, w2, "second call")
     # and once more on the first context (second outer iteration, non-zero slow momentum)
     _one_call(s1, w1, "third call")
+    # a call that only enqueues (wait = 0), followed by a waiting one that reuses the scratch
+    _one_call(s2, w2, "fourth call, not waiting", wait=False)
+    _one_call(s1, w1, "fifth call")
     s1.close()
     s2.close()
 
