@@ -5,15 +5,24 @@ bandwidth of the fused local-step and outer-step kernels.
     python bench.py --gpus N --steps K --warmup W            (this library)
     python bench.py --impl reference --steps K --warmup W    (the CPU oracle, as it stands)
 
-One step = one outer iteration of Algorithm 1 on the ResNet-50-shaped workload: tau fused
-local-step launches over the [m, P] replica tensor and one fused outer-step launch. With
-N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the
-workload on its own GPU: the path has no exchange step, so no collective is on the data
-path; ranks only agree on the slowest time.
+One step = one outer iteration of Algorithm 1 on the largest workload, the bandwidth stress
+(P = 1e9 parameters, m = 4 workers, tau = 12, supplied gradient, 56 GB resident): tau fused
+local-step launches over the [m, P] replica tensor and one fused outer-step launch. The headline
+runs the byte-saving variant of the same step (last inner step inside the outer-step kernel,
+broadcast left to the next iteration's first step); the plain tau + 1 launches are timed in the
+same run and reported beside it, and so are the other workloads (ResNet-50-shaped, BMUF,
+transformer-shaped with Adam, tau = 1 and tau = 48).
+
+With N > 1 every rank runs an independent replica of the workload on its own GPU: the path has no
+exchange step, so no collective is on the data path; ranks only agree on the slowest time. Started
+without a launcher, `--gpus N` starts the N ranks itself (torch.distributed.run on 127.0.0.1).
 """
 import argparse
+import glob
 import json
 import os
+import re
+import socket
 import sys
 import threading
 import time
@@ -26,15 +35,7 @@ METRIC = "replica-param updates/sec (local + outer step)"
 UNIT = "updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch divided by the
-# algorithmic bytes, from ncu captures of small cases of the current kernels (profiles/);
-# traffic grows in proportion to m*P, so the ratio carries to the full launch. None = no capture
-# of the kernel as it stands.
-NCU_TRAFFIC_RATIO = {("local_step", "generated"): 0.961, ("local_step", "supplied"): 0.980,
-                     ("outer_step", "average"): 0.952, ("outer_step", "reset"): 0.973,
-                     ("last_step_outer", "generated-average"): 0.975, ("last_step_outer", "supplied-reset"): 0.983,
-                     ("last_step_outer", "lazy-generated-average"): 1.001, ("last_step_outer", "lazy-supplied-reset"): 0.994,
-                     ("local_step", "virt-generated-average"): 0.940, ("local_step", "virt-supplied-reset"): 0.970}
+HEADLINE = "stress_tau12"
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -53,9 +54,12 @@ def local_step_bytes(w):
 def outer_step_bytes(w):
     """Algorithmic HBM bytes of one fused outer-step launch: m rows read and written, anchor
     and u read and written, plus the buffer policy (reset: nb*m rows written; average: nb*m
-    rows read and written)."""
+    rows read and written). Without the exact average (Section 6): x, anchor, u of every worker
+    read and written, plus the reset rows."""
     m, P = w["m"], w["P"]
     nb = 2 if "adam" in w["base"] else 1
+    if w.get("no_average"):
+        return (24 + (4 * nb if w["buffer_policy"] == "reset" else 0)) * m * P
     per_param = 8 * m + 16
     if w["buffer_policy"] == "reset":
         per_param += 4 * m * nb
@@ -116,6 +120,39 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return FALLBACK_HBM_GBS, "fallback"
+
+
+_TRAFFIC = None
+
+
+def traffic_ratios():
+    """DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch divided by the
+    algorithmic bytes, per kernel case, read from the ncu summaries under profiles/: every line
+    `traffic_ratio: case=<kernel case> ... ratio=<r> source=<hash of the kernel sources>`. A ratio
+    counts only while the kernel sources are the ones the capture was taken on; otherwise the
+    kernel has changed since and the traffic is reported as null."""
+    global _TRAFFIC
+    if _TRAFFIC is None:
+        _TRAFFIC = {}
+        now = kernel_source_hash()
+        for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+            for line in open(path):
+                if line.startswith("traffic_ratio:"):
+                    kv = dict(p.split("=", 1) for p in line.split()[1:] if "=" in p)
+                    if kv.get("source") == now:
+                        _TRAFFIC[kv["case"]] = (float(kv["ratio"]), os.path.basename(path))
+    return _TRAFFIC
+
+
+def kernel_source_hash():
+    """Short hash of the CUDA sources: ties an ncu summary to the kernels it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1910_00643_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        if f.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(csrc, f), "rb").read())
+    return h.hexdigest()[:12]
 
 
 # ------------------------------------------------------------------------------ clock sampling
@@ -206,14 +243,60 @@ def aggregate_throughput(units_this_rank, ms_this_rank, device=None):
     return units / (ms * 1e-3), ms
 
 
+def free_port():
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_command(n_ranks, argv):
+    """The launcher command that starts n_ranks copies of this script on one node."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_ranks}",
+            "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+
+
+def ensure_ranks(args):
+    """`--gpus N` without a launcher: start the N ranks and hand over to them. Under a launcher the
+    rank count must agree with --gpus."""
+    world = os.environ.get("WORLD_SIZE")
+    if world is None:
+        if args.gpus > 1:
+            os.execv(sys.executable, spawn_command(args.gpus, sys.argv[1:]))
+        return
+    if int(world) != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started WORLD_SIZE={world} ranks")
+
+
+def init_process_group(backend, local_rank):
+    """Rendezvous of the ranks started by a launcher; NCCL's banner is kept off stdout, which
+    carries the one JSON line only."""
+    import torch
+    import torch.distributed as dist
+    sys.stdout.flush()
+    saved = os.dup(1)
+    os.dup2(2, 1)
+    try:
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+            dist.barrier()
+            torch.cuda.synchronize()
+        else:
+            dist.init_process_group("gloo")
+            dist.barrier()
+    finally:
+        os.dup2(saved, 1)
+        os.close(saved)
+
+
 # --------------------------------------------------------------------------------- timed loops
 
 def time_steps(s, w, steps, warmup, grad=None, fused=False, lazy=False):
-    """Device-timed outer iterations. Returns total ms and the per-kernel mean launch ms.
-    With the fused variant the last inner step runs inside the outer-step kernel, so an
-    iteration has tau-1 local-step launches. With the lazy variant the first launch of an
-    iteration (which reads the anchor instead of the rows) is timed apart and returned in
-    time_steps.first_ms; the run ends with slowmo_materialize inside the timed region."""
+    """Device-timed outer iterations. Returns total ms, the per-kernel mean launch ms of the local
+    step and of the outer step, and (lazy variant) of the first local step of an iteration.
+    With the fused variant the last inner step runs inside the outer-step kernel, so an iteration
+    has tau-1 local-step launches. With the lazy variant the first launch of an iteration (which
+    reads the anchor instead of the rows) is timed apart; the run ends with slowmo_materialize
+    inside the timed region."""
     import torch
     tau = w["tau"]
     split_first = lazy and tau >= 3
@@ -241,11 +324,11 @@ def time_steps(s, w, steps, warmup, grad=None, fused=False, lazy=False):
     torch.cuda.synchronize()
     barrier()
     total = ev[0][0].elapsed_time(end)
-    time_steps.first_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / steps if split_first else None
-    local = sum(e[1].elapsed_time(e[2]) for e in ev) / (steps * local_launches)
+    first = sum(e[0].elapsed_time(e[1]) for e in ev) / steps if split_first else None
+    local = sum(e[1].elapsed_time(e[2]) for e in ev) / (steps * local_launches) if not (fused and tau == 1) else None
     outer = sum(e[2].elapsed_time(e[3]) for e in ev) / steps
     s.sync_status()
-    return total, local, outer
+    return total, local, outer, first
 
 
 def time_steps_e2e(s, w, steps, warmup, host_in, host_out, chunks=16):
@@ -254,9 +337,12 @@ def time_steps_e2e(s, w, steps, warmup, host_in, host_out, chunks=16):
     import torch
 
     def one():
-        # H2D of the [m, P] centres, tau local steps + outer step, D2H of the new outer iterate,
+        # H2D of the [m, P] input, tau local steps + outer step, D2H of the new outer iterate,
         # pipelined over column windows inside the library call
-        s.iteration_host(host_in, host_out, chunks)
+        if w["grad_mode"] == "generated":
+            s.iteration_host(host_in, host_out, chunks)
+        else:
+            s.iteration_host_supplied(host_in, host_out, chunks)
 
     for _ in range(warmup):
         one()
@@ -279,84 +365,112 @@ def time_steps_e2e(s, w, steps, warmup, host_in, host_out, chunks=16):
 
 def roofline(kind, bytes_per_launch, ms, peak, peak_kind, case=None):
     achieved = bytes_per_launch / (ms * 1e-3) / 1e9
-    ratio = NCU_TRAFFIC_RATIO.get((kind, case))
+    ratio, source = traffic_ratios().get(case, (None, None))
     return {"bound": "hbm", "kernel": kind, "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
             "frac": round(achieved / peak, 4), "peak_kind": peak_kind + " copy bandwidth",
             "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
             "bytes_per_launch": bytes_per_launch, "ms_per_launch": round(ms, 4),
             "traffic": None if ratio is None else int(ratio * bytes_per_launch),
             "traffic_source": None if ratio is None else
-            f"ncu small-case capture scaled by m*P (traffic / algorithmic = {ratio})"}
+            f"profiles/{source}: ncu small-case capture scaled by m*P (traffic / algorithmic = {ratio})",
+            "case": case}
 
 
-def cpu_baseline(w, budget_s=15.0):
-    """The oracle, untouched, on a contiguous slice of the same workload sized for ~budget_s."""
-    import oracle
-    cfg = oracle.make_config(**w)
-    n0 = 512
-    t0 = time.perf_counter()
-    oracle.run(cfg, j0=0, n=n0, precision="f32")
-    dt = max(time.perf_counter() - t0, 1e-4)
-    n = int(max(n0, min(w["P"], n0 * budget_s / dt)))
-    t0 = time.perf_counter()
-    oracle.run(cfg, j0=0, n=n, precision="f32")
-    dt = time.perf_counter() - t0
-    updates = n * w["m"] * w["tau"] * w["T"]
-    return {"value": updates / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-            "sample": f"coordinates 0..{n - 1} of P={w['P']}, all m={w['m']} workers, tau={w['tau']}, "
-                      f"T={w['T']} outer iterations, binary32 mode, {dt:.1f} s"}
+def kernel_case(w, kernel, variant):
+    """Name of the kernel case as the ncu summaries under profiles/ key it."""
+    base = "adam" if "adam" in w["base"] else "nesterov"
+    if w["base"].startswith("sgp"):
+        return f"sgp_step:{base}:{w['grad_mode']}"
+    if kernel == "local_step":
+        return f"local_step:{base}:{w['grad_mode']}"
+    if kernel == "first_local_step":
+        return f"local_step_virtual:{base}:{w['grad_mode']}:{w['buffer_policy']}"
+    if w.get("no_average"):
+        return f"outer_step_noaverage:{base}:{w['buffer_policy']}"
+    if variant in ("fused", "lazy"):
+        return f"last_step_outer_{variant}:{base}:{w['grad_mode']}:{w['buffer_policy']}"
+    return f"outer_step_{variant}:{base}:{w['buffer_policy']}"
 
 
-def stress_extra(peak, peak_kind, tau=12, iters=2):
-    """Largest configuration (supplied gradient, P = 1e9, m = 4): per-kernel bandwidth."""
+def measure(name, variant, steps, warmup, peak, peak_kind, overrides=None, context=None):
+    """One workload in one outer-step variant: whole-step time and per-kernel rooflines. Returns
+    (result dict, context) — the context is kept open when `context` was given or asked for."""
     import torch
     from paper_1910_00643_b200 import SlowMo, workloads
-    w = workloads.workload("stress_tau12", tau=tau)
-    out = {"workload": "stress P=1e9 m=4 supplied gradient"}
-    s = SlowMo(w)
-    s.alloc_gradient()
-    s.fill_gradient()
-    for variant in ("direct", "staged", "fused", "lazy"):
-        s.set_variant("outer", variant)
-        total, local, outer = time_steps(s, w, iters, 1, s.grad, fused=variant in ("fused", "lazy"),
-                                         lazy=variant == "lazy")
-        if variant == "lazy":
-            out["last_step_outer_lazy"] = roofline("last_step_outer", lazy_outer_step_bytes(w), outer, peak, peak_kind,
-                                                   "lazy-supplied-reset")
-            out["first_local_step_lazy"] = roofline("local_step", virtual_first_step_bytes(w), time_steps.first_ms,
-                                                    peak, peak_kind, "virt-supplied-reset")
-        elif variant == "fused":
-            out["last_step_outer_fused"] = roofline("last_step_outer", fused_outer_step_bytes(w), outer, peak,
-                                                    peak_kind, "supplied-reset")
-        else:
-            out["local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind, "supplied")
-            out["outer_step_" + variant] = roofline("outer_step", outer_step_bytes(w), outer, peak, peak_kind,
-                                                    "reset" if variant == "direct" else None)
-        out["updates_per_s_tau%d_%s" % (tau, variant)] = w["m"] * w["P"] * tau * iters / (total * 1e-3)
+    w = workloads.workload(name, **(overrides or {}))
+    s = context if context is not None else SlowMo(w)
+    if context is None and w["grad_mode"] == "supplied":
+        s.alloc_gradient()
+        s.fill_gradient()
+    s.set_variant("outer", variant)
+    plain = w["base"].startswith("sgp") or w.get("no_average")
+    fused = variant in ("fused", "lazy") and not plain
+    lazy = fused and variant == "lazy" and w["tau"] >= 2
+    total, local, outer, first = time_steps(s, w, steps, warmup, s.grad, fused=fused, lazy=lazy)
+    out = {"workload": name, "outer_variant": variant, "steps": steps,
+           "ms_per_step": round(total / steps, 4), "value": w["m"] * w["P"] * w["tau"] * steps / (total * 1e-3),
+           "unit": UNIT, "launches_per_step": w["tau"] + (0 if fused else 1)}
+    if local is not None:
+        out["roofline_local_step"] = roofline("local_step", local_step_bytes(w), local, peak, peak_kind,
+                                              kernel_case(w, "local_step", variant))
+    nbytes = lazy_outer_step_bytes(w) if lazy else fused_outer_step_bytes(w) if fused else outer_step_bytes(w)
+    out["roofline_outer_step"] = roofline("last_step_outer" if fused else "outer_step", nbytes, outer, peak, peak_kind,
+                                          kernel_case(w, "outer_step", variant if (fused or not plain) else "direct"))
+    if first is not None:
+        out["roofline_first_local_step"] = roofline("local_step", virtual_first_step_bytes(w), first, peak, peak_kind,
+                                                    kernel_case(w, "first_local_step", variant))
+    return out, s, w
+
+
+def release(s):
+    import torch
     s.close()
     del s
     torch.cuda.empty_cache()
-    # the workload is defined as a sweep over tau: whole-run updates/s at tau = 1 and 48 too (T = 3)
-    sweep = {str(tau): {v: out["updates_per_s_tau%d_%s" % (tau, v)] for v in ("direct", "fused", "lazy")}}
-    for t_in in (1, 48):
-        wt = workloads.workload("stress_tau12", tau=t_in)
-        s = SlowMo(wt)
-        s.alloc_gradient()
-        s.fill_gradient()
-        sweep[str(t_in)] = {}
-        for variant in ("direct", "fused", "lazy"):
-            s.set_variant("outer", variant)
-            total, _, _ = time_steps(s, wt, wt["T"], 1, s.grad, fused=variant in ("fused", "lazy"),
-                                     lazy=variant == "lazy")
-            sweep[str(t_in)][variant] = wt["m"] * wt["P"] * t_in * wt["T"] / (total * 1e-3)
-        s.close()
-        del s
-        torch.cuda.empty_cache()
-    out["updates_per_s_by_tau"] = sweep
-    return out
+
+
+def cpu_baseline(w, budget_s=12.0):
+    """The oracle, untouched, on a contiguous slice of the same workload: once on all host cores
+    (the headline `value`), once on a single thread, each sized for about budget_s seconds."""
+    import oracle
+    cfg = oracle.make_config(**w)
+    per_coord = w["m"] * w["tau"] * w["T"]
+
+    def timed(threads):
+        # grow the slice until a run takes long enough to extrapolate from, then size it for the budget
+        n, dt = 4096, 0.0
+        while True:
+            t0 = time.perf_counter()
+            oracle.run(cfg, j0=0, n=n, precision="f32", threads=threads)
+            dt = time.perf_counter() - t0
+            if dt >= 0.5 or n >= w["P"]:
+                break
+            n = min(w["P"], n * 8)
+        n = int(max(4096, min(w["P"], 1 << 26, n * budget_s / max(dt, 1e-3))))
+        t0 = time.perf_counter()
+        oracle.run(cfg, j0=0, n=n, precision="f32", threads=threads)
+        dt = time.perf_counter() - t0
+        return n * per_coord / dt, n, dt
+
+    cores = oracle.threads()
+    v_all, n_all, dt_all = timed(None)
+    v_one, n_one, dt_one = timed(1)
+    what = f"all m={w['m']} workers, tau={w['tau']}, T={w['T']} outer iterations, binary32 mode"
+    return {"value": v_all, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"coordinates 0..{n_all - 1} of P={w['P']}, {what}, {dt_all:.1f} s on {cores} threads",
+            "single_thread": {"value": v_one, "unit": UNIT, "cores": 1,
+                              "sample": f"coordinates 0..{n_one - 1} of P={w['P']}, {what}, {dt_one:.1f} s on 1 thread"}}
 
 
 # -------------------------------------------------------------------------------------- arms
+
+def host_memory_available():
+    try:
+        import psutil
+        return psutil.virtual_memory().available
+    except Exception:
+        return 0
+
 
 def size_overrides(args):
     """Optional smaller problem (for profiler captures); the default is the named workload."""
@@ -369,115 +483,206 @@ def size_overrides(args):
     return over
 
 
+def describe(w, name):
+    return (f"{name}: P={w['P']} m={w['m']} tau={w['tau']} base={w['base']} buffers={w['buffer_policy']} "
+            f"grad={w['grad_mode']}")
+
+
+STEP_TEXT = {
+    "lazy": "one outer iteration = tau-1 local-step launches (the first reads the anchor in place of the replica "
+            "rows) + one launch of the outer step with the last inner step fused in and the broadcast left to the "
+            "next iteration (SLOWMO_OUTER_LAZY); the timed region ends with slowmo_materialize",
+    "fused": "one outer iteration = tau-1 local-step launches + one launch of the outer step with the last inner "
+             "step fused in (SLOWMO_OUTER_FUSED)",
+    "direct": "one outer iteration = tau local-step launches + one outer-step launch",
+    "staged": "one outer iteration = tau local-step launches + one outer-step launch (bulk-copy staging)",
+}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_1910_00643_b200 import SlowMo, workloads
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
-    launched = "RANK" in os.environ and "MASTER_ADDR" in os.environ   # under torch.distributed.run
-    if world > 1 or launched:
-        # NCCL announces its version on stdout when the communicator is created: send that to
-        # stderr so that stdout carries the one JSON line only
-        sys.stdout.flush()
-        saved = os.dup(1)
-        os.dup2(2, 1)
-        try:
-            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-            dist.barrier()
-            torch.cuda.synchronize()
-        finally:
-            os.dup2(saved, 1)
-            os.close(saved)
+    if world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ):   # under a launcher
+        init_process_group("nccl", local_rank)
     dev = torch.device("cuda", local_rank)
-
-    w = workloads.workload(args.workload, **size_overrides(args))
     peak, peak_kind = measured_peak()
-    s = SlowMo(w)
-    s.set_variant("outer", args.outer_variant)
-    fused = (args.outer_variant in ("fused", "lazy") and (w["grad_mode"] == "supplied" or w["m"] <= 64)
-             and w["tau"] > 1 and not w["base"].startswith("sgp") and not w.get("no_average"))
-    lazy = fused and args.outer_variant == "lazy"
-    grad = None
-    if w["grad_mode"] == "supplied":
-        grad = s.alloc_gradient()
-        s.fill_gradient()
+    over = size_overrides(args)
+    name, variant = args.workload, args.outer_variant
 
+    # ---- headline: device-resident, timed between barriers, clocks sampled meanwhile
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, local_ms, outer_ms = time_steps(s, w, args.steps, args.warmup, grad, fused=fused, lazy=lazy)
-    first_ms = time_steps.first_ms
+    head, s, w = measure(name, variant, args.steps, args.warmup, peak, peak_kind, over)
     clocks = sampler.stop()
-    units = w["m"] * w["P"] * w["tau"] * args.steps
-    value, ms = aggregate_throughput(units, total_ms, dev)
+    value, ms = aggregate_throughput(w["m"] * w["P"] * w["tau"] * args.steps, head["ms_per_step"] * args.steps, dev)
 
-    # end to end: host buffers in and out through the C ABI
+    # ---- the plain tau + 1 launches of the same workload, same context, same run
+    plain = None
+    if variant != "direct" and not args.no_extra:
+        plain, _, _ = measure(name, "direct", max(2, args.steps // 4), 1, peak, peak_kind, over, context=s)
+        staged, _, _ = measure(name, "staged", 2, 1, peak, peak_kind, over, context=s)
+        plain["roofline_outer_step_staged"] = staged["roofline_outer_step"]
+        s.set_variant("outer", variant)
+
+    # ---- end to end: host buffers in and out through the C ABI
     e2e = None
-    if w["grad_mode"] == "generated" and not args.no_e2e:
+    host_bytes = 4 * (w["m"] + 1) * w["P"]
+    if not args.no_e2e and host_memory_available() < 2 * host_bytes:
+        e2e = {"skipped": f"needs {host_bytes / 1e9:.1f} GB of pinned host memory; "
+                          f"{host_memory_available() / 1e9:.1f} GB available"}
+    elif not args.no_e2e:
+        generated = w["grad_mode"] == "generated"
         host_in = torch.empty((w["m"], w["P"]), dtype=torch.float32, pin_memory=True)
         host_out = torch.empty((1, w["P"]), dtype=torch.float32, pin_memory=True)
-        s.get_params("c", out=host_in)  # the same per-worker data the device-resident run used
-        e2e_steps = max(1, min(args.steps, 5))
+        # the same per-worker data the device-resident run used
+        if generated:
+            s.get_params("c", out=host_in)
+        else:
+            s.synchronize()
+            host_in.copy_(s.grad.view(w["m"], s.pitch)[:, :w["P"]])
+        e2e_steps = max(1, min(args.steps, 4))
         e2e_ms = time_steps_e2e(s, w, e2e_steps, 1, host_in, host_out)
         e2e_value, _ = aggregate_throughput(w["m"] * w["P"] * w["tau"] * e2e_steps, e2e_ms, dev)
         e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": host_in.numel() * 4,
                "d2h_bytes_per_step": host_out.numel() * 4, "steps": e2e_steps,
                "ms_per_step": round(e2e_ms / e2e_steps, 3),
-               "note": "each step is one slowmo_iteration_host call: uploads the per-worker centres c [m,P] "
-                       "from pinned host memory and reads x_{t+1,0} back, pipelined with the kernels over "
-                       "16 column windows"}
+               "note": "each step is one slowmo_iteration_host%s call: uploads the per-worker %s [m,P] from pinned "
+                       "host memory and reads x_{t+1,0} back, pipelined with the kernels over 16 column windows"
+                       % ("" if generated else "_supplied", "centres c" if generated else "gradient G")}
         del host_in, host_out
-    s.close()
-    del s
-    torch.cuda.empty_cache()
+    release(s)
 
+    fused = head["launches_per_step"] == w["tau"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: P={w['P']} m={w['m']} tau={w['tau']} "
-                               f"base={w['base']} buffers={w['buffer_policy']} grad={w['grad_mode']}",
-                   "step": ("one outer iteration = tau-1 local-step launches (the first reads the anchor in "
-                            "place of the replica rows) + one launch of the outer step with the last inner "
-                            "step fused in and the broadcast left to the next iteration (SLOWMO_OUTER_LAZY); "
-                            "the timed region ends with slowmo_materialize") if lazy else
-                           ("one outer iteration = tau-1 local-step launches + one launch of the outer step "
-                            "with the last inner step fused in (SLOWMO_OUTER_FUSED)") if fused else
-                           "one outer iteration = tau local-step launches + one outer-step launch",
-                   "outer_variant": args.outer_variant,
+        "config": {"workload": describe(w, name), "step": STEP_TEXT[variant if fused or variant == "staged" else "direct"],
+                   "outer_variant": variant,
                    "replicas": "independent replica of the workload per GPU, no collective on the data path",
-                   "l2": "state tensors (>= 5 GB) are far larger than the 126 MB L2; no flush needed"},
-        "gpu_launches": args.steps * (w["tau"] + (0 if fused else 1)) + (1 if lazy else 0),
+                   "l2": "state tensors (56 GB at the default workload) are far larger than the 126 MB L2; no flush needed"},
+        "gpu_launches": args.steps * head["launches_per_step"] + (1 if variant == "lazy" and fused else 0),
         "clocks": clocks,
-        "roofline": roofline("local_step", local_step_bytes(w), local_ms, peak, peak_kind,
-                             w["grad_mode"] if w["base"] == "nesterov" else None),
-        "roofline_outer_step": (
-            roofline("last_step_outer", lazy_outer_step_bytes(w), outer_ms, peak, peak_kind,
-                     f"lazy-{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if lazy else
-            roofline("last_step_outer", fused_outer_step_bytes(w), outer_ms, peak, peak_kind,
-                     f"{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None) if fused else
-            roofline("outer_step", outer_step_bytes(w), outer_ms, peak, peak_kind,
-                     w["buffer_policy"] if args.outer_variant == "direct" and w["base"] == "nesterov"
-                     and w["buffer_policy"] != "maintain" else None)),
+        "roofline": head.get("roofline_local_step") or head["roofline_outer_step"],
+        "roofline_outer_step": head["roofline_outer_step"],
         "e2e": e2e,
     }
-    if lazy and first_ms is not None:
-        line["roofline_first_local_step"] = roofline(
-            "local_step", virtual_first_step_bytes(w), first_ms, peak, peak_kind,
-            f"virt-{w['grad_mode']}-{w['buffer_policy']}" if w["base"] == "nesterov" else None)
+    if "roofline_first_local_step" in head:
+        line["roofline_first_local_step"] = head["roofline_first_local_step"]
+    if plain is not None:
+        line["direct_variant"] = plain
     if rank == 0 and world == 1:
-        if not args.no_stress:
-            try:
-                line["stress"] = stress_extra(peak, peak_kind)
-            except Exception as exc:  # out of memory on a smaller device: report, do not hide
-                line["stress"] = {"error": repr(exc)}
+        if not args.no_extra:
+            line["other_workloads"] = other_workloads(peak, peak_kind, skip=name)
         if not args.no_cpu:
-            line["cpu_baseline"] = cpu_baseline(w, args.cpu_seconds)
+            from paper_1910_00643_b200 import workloads
+            line["cpu_baseline"] = cpu_baseline(workloads.workload(name, **over), args.cpu_seconds)
     if rank == 0:
         print(json.dumps(line))
+    if dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def other_workloads(peak, peak_kind, skip):
+    """The remaining workloads, a few outer iterations each, in the lazy and the direct variant."""
+    out = {}
+    for name, steps in (("stress_tau1", 3), ("stress_tau48", 2), ("resnet50", 5), ("bmuf", 2), ("transformer_adam", 3)):
+        if name == skip:
+            continue
+        try:
+            res, s, _ = measure(name, "lazy", steps, 1, peak, peak_kind)
+            direct, _, _ = measure(name, "direct", steps, 1, peak, peak_kind, context=s)
+            release(s)
+            res["direct_variant"] = direct
+            out[name] = res
+        except Exception as exc:  # e.g. out of memory on a smaller device: report, do not hide
+            out[name] = {"error": repr(exc)}
+    return out
+
+
+def run_sharded(args):
+    """Workers sharded over the GPUs (one process per GPU, m / N workers each): the local steps run on
+    each GPU's own rows and the outer step is slowmo_outer_step_sharded, which does the exact average
+    over peer-mapped memory. Reports the step time, the outer step's share of it and the NVLink bytes
+    each GPU moves per outer step, beside the expectation (1 - 1/N) * m * (P/N) * 4 bytes each way
+    for the x rows (buffer rows on top under the average policy)."""
+    import torch
+    import torch.distributed as dist
+    from paper_1910_00643_b200 import workloads
+    from paper_1910_00643_b200.sharded import ShardedSlowMo
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if "RANK" not in os.environ:       # one rank without a launcher still needs a process group
+        os.environ.update(RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(free_port()))
+    os.environ.setdefault("NCCL_NVLS_ENABLE", "0")   # peer memory is touched with plain loads and stores only
+    init_process_group("nccl", local_rank)
+    dev = torch.device("cuda", local_rank)
+    name = "resnet50" if args.workload == HEADLINE else args.workload
+    w = workloads.workload(name, **size_overrides(args))
+    s = ShardedSlowMo(w)
+    tau, steps = w["tau"], args.steps
+    for _ in range(args.warmup):
+        s.local_steps(tau)
+        s.outer_step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    s.local.synchronize()
+    barrier()
+    torch.cuda.synchronize()
+    for i in range(steps):
+        ev[i][0].record(s.local.stream)
+        s.local_steps(tau)
+        ev[i][1].record(s.local.stream)
+        s.outer_step()                     # fence, sharded kernel, fence
+        ev[i][2].record(s.local.stream)
+    s.local.synchronize()
+    torch.cuda.synchronize()
+    barrier()
+    total = ev[0][0].elapsed_time(ev[-1][2])
+    outer = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+    value, ms = aggregate_throughput(s.m_local * w["P"] * tau * steps, total, dev)
+    outer_ms = max_over_ranks(outer, dev)
+    nb = 2 if "adam" in w["base"] else 1
+    rows = 1 + (nb if w["buffer_policy"] == "average" else 0)          # row sets read from peers
+    wrows = 1 + (nb if w["buffer_policy"] != "maintain" else 0)        # row sets written to peers
+    slice_cols = w["P"] / world
+    remote = (world - 1) * s.m_local * slice_cols * 4
+    line = {"mode": "sharded", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": args.warmup, "ms_per_step": round(ms / steps, 4), "higher_is_better": True, "scaling": "strong",
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w, name), "workers_per_gpu": s.m_local,
+                       "step": "tau local-step launches on each GPU's own rows + fence + one sharded outer-step kernel "
+                               "per GPU (reduce-scatter, Eq. 2/3, all-gather over peer memory) + fence"},
+            "outer_step_ms": round(outer_ms, 4), "outer_step_share": round(outer_ms * steps / ms, 4),
+            "nvlink_bytes_per_gpu_per_outer_step": {
+                "read_from_peers": int(rows * remote), "written_to_peers": int(wrows * remote + (world - 1) * 8 * slice_cols),
+                "expected_for_x_rows_each_way": int(remote),
+                "formula": "(1 - 1/N) * m * (P/N) * 4 bytes for each set of rows read or written, plus the anchor and u "
+                           "slices written to every peer"},
+            "peer_access": "plain loads and stores; no bulk copy, no multicast, no library kernel on peer memory"}
+    s.close()
+    if rank == 0:
+        print(json.dumps(line))
+    dist.destroy_process_group()
+
+
+def run_selftest_ranks(args):
+    """Host-only check of the rank plumbing (no GPU): gloo rendezvous, aggregation, one JSON line."""
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    if "RANK" in os.environ:
+        init_process_group("gloo", 0)
+    value, ms = aggregate_throughput(1000.0 * (rank + 1), 10.0 * (rank + 1))
+    barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": "ranks", "n_gpus": world, "value": value, "ms": ms}))
     if dist.is_initialized():
         dist.destroy_process_group()
 
@@ -506,8 +711,7 @@ def run_reference(args):
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: P={w['P']} m={w['m']} tau={w['tau']} base={w['base']} "
-                               f"buffers={w['buffer_policy']} grad={w['grad_mode']}", "sample": sample},
+        "config": {"workload": describe(w, args.workload), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -520,20 +724,33 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet50")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "sharded"],
+                    help="replicas: every GPU runs the whole workload (the default). sharded: the m workers of "
+                         "the ResNet-50-shaped workload are spread over the GPUs and the outer step averages "
+                         "over peer memory")
+    ap.add_argument("--workload", default=HEADLINE)
     ap.add_argument("--outer-variant", default="lazy", choices=["direct", "staged", "fused", "lazy"])
     ap.add_argument("--P", type=int, default=None, help="override the workload's parameter count")
     ap.add_argument("--m", type=int, default=None, help="override the workload's worker count")
     ap.add_argument("--tau", type=int, default=None, help="override the workload's inner steps")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
-    ap.add_argument("--no-stress", action="store_true", help="skip the P=1e9 per-kernel measurement")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the direct-variant figure of the same workload and the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
-    ap.add_argument("--cpu-seconds", type=float, default=15.0)
-    ap.add_argument("--reference-coords", type=int, default=1 << 17)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--reference-coords", type=int, default=1 << 20)
+    ap.add_argument("--selftest-ranks", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
+    ensure_ranks(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.impl == "reference":
+    if args.selftest_ranks:
+        run_selftest_ranks(args)
+    elif args.impl == "reference":
         run_reference(args)
+    elif args.mode == "sharded":
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -221,6 +221,18 @@ int slowmo_outer_step(slowmo_ctx *ctx);
 int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks);
 
 /*
+ * The same for supplied-gradient mode (ENOTIMPL otherwise): the stochastic gradients of the
+ * iteration, grad_host [m, P] (dense, host, pinned for overlap), are uploaded window by window into
+ * the caller's DEVICE staging tensor grad_dev [m, pitch] (16-byte aligned, borrowed for the call),
+ * and each window's tau local steps read it there, as slowmo_local_steps(tau, grad_dev) would: the
+ * same gradient at each of the tau steps (Algorithm 1's stochastic gradient, held fixed over the
+ * iteration). Bit-identical to copying grad_host into grad_dev and calling
+ * slowmo_local_steps(tau, grad_dev) + slowmo_outer_step + slowmo_get_params(anchor).
+ */
+int slowmo_iteration_host_supplied(slowmo_ctx *ctx, const float *grad_host, float *grad_dev, float *anchor_host,
+                                   uint32_t chunks);
+
+/*
  * Outer step of Algorithm 1 for workers sharded over several GPUs of one node: the exact average
  * (the paper's AllReduce) fused with Eq. (2), Eq. (3), the broadcast and the buffer policy in
  * one kernel per GPU that reads and writes the other GPUs' memory directly.

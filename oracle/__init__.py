@@ -65,6 +65,8 @@ def lib():
         L.oracle_centre.argtypes = [C.POINTER(_Cfg), C.c_uint32, C.c_uint64]
         L.oracle_supplied_gradient.argtypes = [C.POINTER(_Cfg), C.c_uint32, C.c_uint64]
         L.slowmo_oracle_threads.restype = C.c_int
+        L.omp_set_num_threads.restype = None       # OpenMP runtime the library is linked with
+        L.omp_set_num_threads.argtypes = [C.c_int]
         L.oracle_sgp_hops.restype = C.c_uint32
         L.oracle_sgp_hops.argtypes = [C.c_uint32, C.c_uint64]
         _lib = L
@@ -85,11 +87,12 @@ def _ptr(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
 
 
-def run(cfg, *, j=None, j0=0, n=None, precision="f32", gamma_t=None, G=None, want_dbar=False):
+def run(cfg, *, j=None, j0=0, n=None, precision="f32", gamma_t=None, G=None, want_dbar=False, threads=None):
     """Run Algorithm 1 on coordinates `j` (uint64 array) or j0..j0+n-1.
 
     Returns dict with x,h,v [m,n], anchor,u [n] (and dbar [T,tau,n] if asked), in float32
-    (precision="f32") or float64 (precision="f64").
+    (precision="f32") or float64 (precision="f64"). `threads` limits the OpenMP threads of this
+    one call (the coordinates are shared out among them; results do not depend on it).
     """
     if not isinstance(cfg, _Cfg):
         cfg = make_config(**cfg)
@@ -112,8 +115,16 @@ def run(cfg, *, j=None, j0=0, n=None, precision="f32", gamma_t=None, G=None, wan
         G = np.ascontiguousarray(G, dtype=np.float32)
         assert G.shape == (cfg.T * cfg.tau, m, n), G.shape
     fn = lib().slowmo_oracle_run_f32 if precision == "f32" else lib().slowmo_oracle_run_f64
-    rc = fn(C.byref(cfg), _ptr(gamma_t), _ptr(j), j0, n, _ptr(G), _ptr(out["x"]),
-            _ptr(out["anchor"]), _ptr(out["u"]), _ptr(out["h"]), _ptr(out["v"]), _ptr(dbar))
+    before = threads_in_use = lib().slowmo_oracle_threads()
+    if threads is not None:
+        lib().omp_set_num_threads(int(threads))
+        threads_in_use = int(threads)
+    try:
+        rc = fn(C.byref(cfg), _ptr(gamma_t), _ptr(j), j0, n, _ptr(G), _ptr(out["x"]),
+                _ptr(out["anchor"]), _ptr(out["u"]), _ptr(out["h"]), _ptr(out["v"]), _ptr(dbar))
+    finally:
+        if threads_in_use != before:
+            lib().omp_set_num_threads(before)
     if rc != 0:
         raise ValueError("oracle rejected the configuration")
     if want_dbar:

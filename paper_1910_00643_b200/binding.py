@@ -26,7 +26,8 @@ EXPORTS = ["slowmo_create", "slowmo_destroy", "slowmo_local_steps", "slowmo_oute
            "slowmo_set_variant", "slowmo_sync_status", "slowmo_strerror", "slowmo_last_cuda_error",
            "slowmo_outer_step_static", "slowmo_debug_wait_timeout", "slowmo_iteration_host", "slowmo_materialize",
            "slowmo_outer_step_sharded", "slowmo_outer_step_external",
-           "slowmo_debug_words_to_normals", "slowmo_get_state", "slowmo_set_state"]
+           "slowmo_debug_words_to_normals", "slowmo_get_state", "slowmo_set_state",
+           "slowmo_iteration_host_supplied"]
 
 
 class SlowMoError(RuntimeError):
@@ -105,6 +106,7 @@ def lib():
             "slowmo_last_cuda_error": [vp],
             "slowmo_debug_wait_timeout": [vp, u32],
             "slowmo_iteration_host": [vp, vp, vp, u32],
+            "slowmo_iteration_host_supplied": [vp, vp, vp, vp, u32],
             "slowmo_materialize": [vp],
             "slowmo_outer_step_sharded": [C.POINTER(ShardArgs), vp],
             "slowmo_outer_step_external": [vp],
@@ -274,6 +276,14 @@ class SlowMo:
         anchor (torch CPU tensors, pinned for overlap, or numpy arrays)."""
         ptr = lambda a: a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
         _check(lib().slowmo_iteration_host(self.ctx, ptr(c_host), ptr(anchor_host), chunks), "slowmo_iteration_host")
+
+    def iteration_host_supplied(self, grad_host, anchor_host, chunks=8, grad_dev=None):
+        """slowmo_iteration_host_supplied: one outer iteration with the host gradient grad_host [m, P]
+        staged through the device tensor grad_dev (default: the context's gradient buffer)."""
+        grad_dev = self.grad if grad_dev is None else grad_dev
+        ptr = lambda a: a.ctypes.data if isinstance(a, np.ndarray) else a.data_ptr()
+        _check(lib().slowmo_iteration_host_supplied(self.ctx, ptr(grad_host), grad_dev.data_ptr(), ptr(anchor_host),
+                                                    chunks), "slowmo_iteration_host_supplied")
 
     def outer_step_external(self):
         _check(lib().slowmo_outer_step_external(self.ctx), "slowmo_outer_step_external")

@@ -455,11 +455,19 @@ int slowmo_outer_step(slowmo_ctx *ctx) {
   return SLOWMO_OK;
 }
 
-int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks) {
-  if (!ctx || !c_host || !anchor_host || chunks == 0 || chunks > 1024) return SLOWMO_EINVAL;
+}  // extern "C"
+
+namespace {
+
+// One whole outer iteration with host input and output, pipelined over column windows. The
+// per-worker input `in_host` [m, P] goes to the device tensor `in_dev` [m, pitch] (the centres c in
+// generated mode, a gradient buffer in supplied mode) window by window; `grad` is what the local
+// steps are given (NULL in generated mode, in_dev in supplied mode).
+int iteration_host(slowmo_ctx *ctx, const float *in_host, float *in_dev, const float *grad, float *anchor_host,
+                   uint32_t chunks) {
+  if (!ctx || !in_host || !in_dev || !anchor_host || chunks == 0 || chunks > 1024) return SLOWMO_EINVAL;
   if (ctx->cuda_error) return SLOWMO_ECUDA;
   const slowmo_config &c = ctx->cfg;
-  if (c.grad_mode != SLOWMO_GRAD_GENERATED) return SLOWMO_ENOTIMPL;
   if (ctx->k != 0 || ctx->pending_last) return SLOWMO_ESTATE;
   cudaError_t e = cudaSuccess;
   if (!ctx->copy_in) e = cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking);
@@ -476,7 +484,7 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
   for (auto &x : ev)
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&x, cudaEventDisableTiming);
   int rc = SLOWMO_OK;
-  // uploads must not overtake earlier work of this context that still reads the centres
+  // uploads must not overtake earlier work of this context that still reads the input tensor
   if (e == cudaSuccess) e = cudaEventRecord(ev[2 * nwin], ctx->stream);
   if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->copy_in, ev[2 * nwin], 0);
 
@@ -487,7 +495,7 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
     const uint32_t vec0 = w * win, nv = ctx->nvec - vec0 < win ? ctx->nvec - vec0 : win;
     const uint64_t col0 = 4ull * vec0;
     const uint64_t cols = c.P - col0 < 4ull * nv ? c.P - col0 : 4ull * nv;  // host arrays have no padding
-    e = cudaMemcpy2DAsync(ctx->buf.c + col0, dpitch, c_host + col0, hpitch, cols * sizeof(float), c.m,
+    e = cudaMemcpy2DAsync(in_dev + col0, dpitch, in_host + col0, hpitch, cols * sizeof(float), c.m,
                           cudaMemcpyHostToDevice, ctx->copy_in);
     if (e == cudaSuccess) e = cudaEventRecord(ev[2 * w], ctx->copy_in);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->stream, ev[2 * w], 0);
@@ -501,7 +509,7 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
     ctx->virt = virt0;
     ctx->win_vec0 = vec0;
     ctx->win_nvec = nv;
-    rc = slowmo_local_steps(ctx, c.tau, nullptr);
+    rc = slowmo_local_steps(ctx, c.tau, grad);
     if (rc == SLOWMO_OK) rc = slowmo_outer_step(ctx);
     if (rc != SLOWMO_OK) break;
     e = cudaEventRecord(ev[2 * w + 1], ctx->stream);
@@ -518,6 +526,24 @@ int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_ho
     if (x) cudaEventDestroy(x);
   if (rc != SLOWMO_OK) return rc;
   return cuda_fail(ctx, e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int slowmo_iteration_host(slowmo_ctx *ctx, const float *c_host, float *anchor_host, uint32_t chunks) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cfg.grad_mode != SLOWMO_GRAD_GENERATED) return SLOWMO_ENOTIMPL;
+  return iteration_host(ctx, c_host, ctx->buf.c, nullptr, anchor_host, chunks);
+}
+
+int slowmo_iteration_host_supplied(slowmo_ctx *ctx, const float *grad_host, float *grad_dev, float *anchor_host,
+                                   uint32_t chunks) {
+  if (!ctx) return SLOWMO_EINVAL;
+  if (ctx->cfg.grad_mode != SLOWMO_GRAD_SUPPLIED) return SLOWMO_ENOTIMPL;
+  if (grad_dev && !aligned16(grad_dev)) return SLOWMO_EALIGN;
+  return iteration_host(ctx, grad_host, grad_dev, grad_dev, anchor_host, chunks);
 }
 
 int slowmo_outer_step_external(slowmo_ctx *ctx) {

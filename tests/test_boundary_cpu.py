@@ -181,6 +181,42 @@ def test_two_rank_aggregation_over_gloo(tmp_path):
         assert "ok" in o
 
 
+def test_gpus_flag_starts_the_ranks_itself(tmp_path):
+    # `bench.py --gpus 2` without a launcher re-executes itself under torch.distributed.run with two
+    # ranks on 127.0.0.1; the host-only self-test stands in for the GPU arm (gloo, no device)
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-ranks"],
+                         capture_output=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr.decode()[-2000:]
+    lines = [l for l in out.stdout.decode().splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout.decode()
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["ms"] == 20.0 and abs(line["value"] - 3000.0 / 0.020) < 1e-6
+    # one rank needs no launcher
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--selftest-ranks"], capture_output=True,
+                         timeout=120, env=env)
+    assert out.returncode == 0 and json.loads(out.stdout.decode().strip())["n_gpus"] == 1
+    # under a launcher that started another number of ranks the mismatch is an error, not a silent 1-GPU run
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-ranks"],
+                         capture_output=True, timeout=120, env=dict(env, WORLD_SIZE="3", RANK="0"))
+    assert out.returncode != 0 and b"WORLD_SIZE=3" in out.stderr
+    import bench
+    cmd = bench.spawn_command(4, ["--gpus", "4", "--steps", "2"])
+    assert "--nproc-per-node=4" in cmd and "127.0.0.1" in cmd and cmd[-4:] == ["--gpus", "4", "--steps", "2"]
+
+
+def test_traffic_ratios_come_from_the_committed_profiles():
+    # every ratio bench.py reports is read from a `traffic_ratio:` line of an ncu summary under profiles/
+    # taken on the current kernel sources; nothing is hard-coded
+    import bench
+    ratios = bench.traffic_ratios()
+    text = "".join(open(os.path.join(ROOT, "profiles", f)).read() for f in os.listdir(os.path.join(ROOT, "profiles")))
+    for case, (ratio, source) in ratios.items():
+        assert f"case={case} " in text and 0.5 < ratio < 1.5 and source.endswith(".md")
+    assert len(bench.kernel_source_hash()) == 12
+
+
 def test_reference_arm_runs_on_the_host():
     out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "1",
                           "--warmup", "0", "--reference-coords", "2048"], capture_output=True, timeout=300)

@@ -126,6 +126,7 @@ sys.path.insert(0, %r)
 import numpy as np, torch, torch.distributed as dist
 rank, world = int(sys.argv[1]), int(sys.argv[2])
 torch.cuda.set_device(rank)
+assert torch.cuda.current_device() == rank        # every rank on a GPU of its own
 os.environ["NCCL_NVLS_ENABLE"] = "0"
 dist.init_process_group("nccl", rank=rank, world_size=world, init_method="tcp://127.0.0.1:" + sys.argv[3],
                         device_id=torch.device("cuda", rank))
@@ -134,8 +135,13 @@ from paper_1910_00643_b200 import workloads
 from paper_1910_00643_b200.sharded import ShardedSlowMo
 w = workloads.workload("tiny", P=5003, m=4, tau=3, T=3, buffer_policy="average", seed=33)
 s = ShardedSlowMo(w)
-s.run(w["T"])
-ref = oracle.run(oracle.make_config(**w), j0=0, n=w["P"], precision="f32")
+assert torch.cuda.current_device() == rank and s.local.t["x"].device.index == rank
+gammas = (w["gamma"] * np.array([1.0, 0.5, 2.0])).astype(np.float32)      # a learning-rate schedule
+for t in range(w["T"]):
+    s.set_gamma(float(gammas[t]))
+    s.local_steps(w["tau"])
+    s.outer_step()
+ref = oracle.run(oracle.make_config(**w), j0=0, n=w["P"], precision="f32", gamma_t=gammas)
 ml = s.m_local
 assert np.array_equal(s.get_params("x").view(np.uint32), ref["x"][rank * ml:(rank + 1) * ml].view(np.uint32))
 assert np.array_equal(s.get_params("h").view(np.uint32), ref["h"][rank * ml:(rank + 1) * ml].view(np.uint32))
