@@ -19,15 +19,14 @@
 
 namespace slowmo {
 
-__device__ __forceinline__ void add_in_order(float4 &s, const float4 &v, bool first) {
-  if (first) {
-    s = v;
-  } else {
-    s.x = __fadd_rn(s.x, v.x);
-    s.y = __fadd_rn(s.y, v.y);
-    s.z = __fadd_rn(s.z, v.z);
-    s.w = __fadd_rn(s.w, v.w);
-  }
+// Running sum over the workers in index order. The sum starts from -0, the one value for which
+// s + v == v bit for bit whatever v is (signed zeros included), so the first worker needs no
+// special case and the result equals x_0 + x_1 + ... added left to right.
+__device__ __forceinline__ float4 ordered_sum_start() { return make_float4(-0.0f, -0.0f, -0.0f, -0.0f); }
+__device__ __forceinline__ void add_in_order(float4 &s, const float4 &v) {
+  const float2 lo = add2(make_float2(s.x, s.y), make_float2(v.x, v.y));
+  const float2 hi = add2(make_float2(s.z, s.w), make_float2(v.z, v.w));
+  s = make_float4(lo.x, lo.y, hi.x, hi.y);
 }
 
 __device__ __forceinline__ float4 div4(const float4 &s, float d) {
@@ -60,7 +59,7 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
   const uint64_t counter = noise_counter(L.vec0 + vi);
   RowKeys<DERIVE> keys;
 
-  float4 sx = a, sh = a, sv = a;  // ordered sums over the workers (overwritten at row 0)
+  float4 sx = ordered_sum_start(), sh = sx, sv = sx;  // ordered sums over the workers
   for (uint32_t i0 = 0; i0 < m; i0 += ROWS) {
     if (GRAD == 0 && (i0 & 31u) == 0) keys.refill(L, i0 + (threadIdx.x & 31u));
     float4 x[ROWS], h[ROWS], v[ROWS], s[ROWS];
@@ -82,18 +81,17 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
       if (GRAD == 0) key = keys.at(L, i, i);
       if (!ok) continue;
       float4 g;
-      if (GRAD == 0) g = generated_gradient(key, counter, a, x[q], s[q], L.sigma);
+      if (GRAD == 0) g = generated_gradient<true>(key, counter, a, x[q], s[q], L.sigma);
       else g = s[q];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
-      add_in_order(sx, x[q], i == 0);
+      base_step4<BASE, GRAD == 0>(L, g, x[q], h[q], v[q]);
+      add_in_order(sx, x[q]);
       if (POLICY == 1) {  // maintain: the stepped buffers go back to their rows
         const uint64_t off = (uint64_t)i * O.pitch + col;
         st_stream(L.h + off, h[q]);
         if (BASE == 1) st_stream(L.v + off, v[q]);
       } else if (POLICY == 2) {  // average
-        add_in_order(sh, h[q], i == 0);
-        if (BASE == 1) add_in_order(sv, v[q], i == 0);
+        add_in_order(sh, h[q]);
+        if (BASE == 1) add_in_order(sv, v[q]);
       }
     }
   }

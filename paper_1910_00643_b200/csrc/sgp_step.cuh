@@ -80,10 +80,9 @@ sgp_step_kernel(const LocalArgs L, uint32_t hops, uint32_t cycles, uint32_t len)
         if (GRAD == 0) key = keys.at(L, n0 + q, i);
         if (!ok) continue;
         float4 g;
-        if (GRAD == 0) g = generated_gradient(key, counter, a, x[q], s[q], L.sigma);
+        if (GRAD == 0) g = generated_gradient<false>(key, counter, a, x[q], s[q], L.sigma);
         else g = s[q];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) base_step<BASE>(L, comp(g, e), comp(x[q], e), comp(h[q], e), comp(v[q], e));
+        base_step4<BASE, false>(L, g, x[q], h[q], v[q]);
         const uint64_t off = (uint64_t)i * L.pitch + col;
         st_stream(L.h + off, h[q]);
         if (BASE == 1) st_stream(L.v + off, v[q]);
