@@ -379,10 +379,8 @@ def roofline(kind, bytes_per_launch, ms, peak, peak_kind, case=None):
 def kernel_case(w, kernel, variant):
     """Name of the kernel case as the ncu summaries under profiles/ key it."""
     base = "adam" if "adam" in w["base"] else "nesterov"
-    if w["base"].startswith("sgp"):
-        return f"sgp_step:{base}:{w['grad_mode']}"
     if kernel == "local_step":
-        return f"local_step:{base}:{w['grad_mode']}"
+        return f"{'sgp_step' if w['base'].startswith('sgp') else 'local_step'}:{base}:{w['grad_mode']}"
     if kernel == "first_local_step":
         return f"local_step_virtual:{base}:{w['grad_mode']}:{w['buffer_policy']}"
     if w.get("no_average"):
@@ -480,6 +478,8 @@ def size_overrides(args):
             over[key] = getattr(args, key)
     if "P" in over:
         over["n_tensors"] = 0
+    if args.no_average:
+        over["no_average"] = True
     return over
 
 
@@ -538,7 +538,7 @@ def run_ours(args):
     elif not args.no_e2e:
         generated = w["grad_mode"] == "generated"
         host_in = torch.empty((w["m"], w["P"]), dtype=torch.float32, pin_memory=True)
-        host_out = torch.empty((1, w["P"]), dtype=torch.float32, pin_memory=True)
+        host_out = torch.empty((w["m"] if w.get("no_average") else 1, w["P"]), dtype=torch.float32, pin_memory=True)
         # the same per-worker data the device-resident run used
         if generated:
             s.get_params("c", out=host_in)
@@ -733,6 +733,8 @@ def main():
     ap.add_argument("--P", type=int, default=None, help="override the workload's parameter count")
     ap.add_argument("--m", type=int, default=None, help="override the workload's worker count")
     ap.add_argument("--tau", type=int, default=None, help="override the workload's inner steps")
+    ap.add_argument("--no-average", action="store_true",
+                    help="run the workload without the exact average (Section 6 of the paper)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the direct-variant figure of the same workload and the other workloads")
