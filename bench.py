@@ -371,6 +371,7 @@ def roofline(kind, bytes_per_launch, ms, peak, peak_kind, case=None):
             "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
             "bytes_per_launch": bytes_per_launch, "ms_per_launch": round(ms, 4),
             "traffic": None if ratio is None else int(ratio * bytes_per_launch),
+            "achieved_dram_traffic": None if ratio is None else round(ratio * achieved, 1),
             "traffic_source": None if ratio is None else
             f"profiles/{source}: ncu small-case capture scaled by m*P (traffic / algorithmic = {ratio})",
             "case": case}

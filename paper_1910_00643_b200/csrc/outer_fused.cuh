@@ -71,7 +71,7 @@ last_step_outer_kernel(const LocalArgs L, const OuterArgs O) {
         h[q] = ld_stream(L.h + off);
         if (BASE == 1) v[q] = ld_stream(L.v + off);
         s[q] = ld_stream(L.src + off);
-        if (prefetch_on<BASE>(SLOWMO_PREFETCH_FUSED) && i0 + q + ROWS < m) {
+        if (prefetch_on<BASE, GRAD>(SLOWMO_PREFETCH_FUSED) && i0 + q + ROWS < m) {
           const uint64_t nxt = off + (uint64_t)ROWS * O.pitch;
           prefetch_l2(L.x + nxt);
           prefetch_l2(L.h + nxt);
