@@ -67,7 +67,7 @@ def _create(binding, buf_overrides=None, **cfg_overrides):
     dict(gamma=float("nan")), dict(beta=1.0), dict(beta=-0.1), dict(alpha=0.0), dict(base=7),
     dict(buffer_policy=3), dict(grad_mode=2), dict(mu=1.0), dict(weight_decay=-1.0),
     dict(base="adam", adam_b1=1.0), dict(base="adam", adam_b2=-0.5), dict(base="adam", adam_eps=0.0),
-    dict(sigma=-1.0), dict(a_lo=2.0, a_hi=1.0), dict(P=2**33), dict(tensor_sizes=[4000, 97]),
+    dict(sigma=-1.0), dict(a_lo=2.0, a_hi=1.0), dict(P=2**33), dict(P=2**32 - 4095), dict(tensor_sizes=[4000, 97]),
     dict(tensor_sizes=[4096, 0]),
 ])
 def test_create_rejects_bad_configurations(binding, bad):

@@ -835,6 +835,36 @@ def test_full_size_with_more_workers_than_inline_noise_keys(layout):
     _free(s)
 
 
+@pytest.mark.parametrize("grad_mode,m,variant,layout", [("generated", 1, "direct", "column_owner"),
+                                                        ("generated", 1, "staged", "row_tiles"),
+                                                        ("supplied", 2, "lazy", "default"),
+                                                        ("supplied", 2, "fused", "default")])
+def test_largest_parameter_count_the_library_accepts(grad_mode, m, variant, layout):
+    # P = 2^32 - 4096 is the largest vector slowmo_create takes (columns are indexed with 32 bits):
+    # rows of 17 GB, 100-140 GB of state. Compared with the oracle at both ends, around the columns whose
+    # byte offsets pass 2^32 and 2^33, in the last tiles, and on sampled coordinates.
+    import torch
+    P = 2**32 - 4096
+    free, _ = torch.cuda.mem_get_info()
+    need = 4 * P * ((3 * m + 3) if grad_mode == "generated" else (3 * m + 2)) + (8 << 30)
+    if free < need:
+        pytest.skip(f"needs {need / 1e9:.0f} GB of device memory, {free / 1e9:.0f} GB free")
+    w = workloads.workload("resnet50", P=P, m=m, tau=2, T=2, n_tensors=0, grad_mode=grad_mode, sigma=0.05)
+    s = _slowmo(w)
+    s.set_variant("outer", variant)
+    s.set_variant("local", layout)
+    grad = None
+    if grad_mode == "supplied":
+        grad = s.alloc_gradient()
+        s.fill_gradient()
+    s.run(2, grad)
+    _check_full_size(s, w, seed=9, slabs=False)
+    near = [np.arange(0, 1 << 16), np.arange(2**30 - 4100, 2**30 + 4100), np.arange(2**31 - 4100, 2**31 + 4100),
+            np.arange(P - (1 << 16), P)]
+    _check_against_oracle(s, w, np.concatenate(near), exact=True)
+    _free(s)
+
+
 def test_full_size_staged_and_fused_outer_steps_equal_direct():
     import torch
     w = workloads.workload("resnet50", T=2)
@@ -858,42 +888,54 @@ FULLP_CHUNK = 1 << 22
 
 
 @pytest.mark.fullp
-@pytest.mark.parametrize("name,variant", [("resnet50", "direct"), ("bmuf", "direct"), ("transformer_adam", "direct"),
-                                          ("stress_tau12", "direct"), ("stress_tau12", "lazy")])
-def test_every_coordinate_of_a_full_size_workload(name, variant):
-    """Selected with -m fullp only (several minutes of oracle time per workload). The device state is
-    brought to the host in chunks of 2^22 coordinates and every element of every state tensor is
-    compared with the oracle bit for bit; the count of coordinates compared and of unequal elements
-    is printed (run with -s) and written to gpurun_out/fullp_<name>_<variant>.txt when that folder exists."""
+@pytest.mark.parametrize("name,variants", [
+    ("resnet50", ("direct", "staged", "fused", "lazy")), ("bmuf", ("direct", "staged", "lazy")),
+    ("local_sgd", ("direct", "lazy")), ("sync_sgd", ("direct", "fused")),
+    ("transformer_adam", ("direct", "fused", "lazy")),
+    ("sgp_resnet50", ("direct",)), ("sgp_transformer_adam", ("direct",)),
+    ("stress_tau1", ("direct", "fused")), ("stress_tau12", ("direct", "lazy")), ("stress_tau48", ("direct", "lazy"))])
+def test_every_coordinate_of_a_full_size_workload(name, variants):
+    """Selected with -m fullp only (minutes of oracle time per workload). Every named variant runs the
+    whole workload on the GPU; then the oracle goes over the vector once, in chunks of 2^22 coordinates,
+    and every element of every state tensor of every variant is compared with it bit for bit. The count
+    of coordinates compared and of unequal elements is printed (run with -s) and written to
+    gpurun_out/fullp_<name>.txt when that folder exists."""
     import os
     import time
     w = workloads.workload(name)
-    s = _slowmo(w)
-    s.set_variant("outer", variant)
-    grad = None
-    if w["grad_mode"] == "supplied":
-        grad = s.alloc_gradient()
-        s.fill_gradient()
-    s.run(w["T"], grad)
-    s.sync_status()
+    runs = []
+    for variant in variants:
+        s = _slowmo(w)
+        s.set_variant("outer", variant)
+        grad = None
+        if w["grad_mode"] == "supplied":
+            grad = s.alloc_gradient()
+            s.fill_gradient()
+        s.run(w["T"], grad)
+        s.sync_status()
+        runs.append(s)
     cfg = oracle.make_config(**w)
-    unequal, compared, t0 = 0, 0, time.time()
+    unequal, compared, t0 = [0] * len(runs), 0, time.time()
     for j0 in range(0, w["P"], FULLP_CHUNK):
         n = min(FULLP_CHUNK, w["P"] - j0)
         ref = oracle.run(cfg, j0=j0, n=n, precision="f32")
-        for key in _state_keys(w):
-            got = s.get_params(key, offset=j0, count=n).reshape(ref[key].shape)
-            unequal += int((got.view(np.uint32) != ref[key].view(np.uint32)).sum())
+        for i, s in enumerate(runs):
+            for key in _state_keys(w):
+                got = s.get_params(key, offset=j0, count=n).reshape(ref[key].shape)
+                unequal[i] += int((got.view(np.uint32) != ref[key].view(np.uint32)).sum())
         compared += n
-    line = (f"{name} ({variant}): {compared} of {w['P']} coordinates compared, all m={w['m']} workers, "
-            f"tensors {','.join(_state_keys(w))}: {unequal} unequal elements, {time.time() - t0:.0f} s")
-    print(line)
+    lines = [f"{name} ({variant}): {compared} of {w['P']} coordinates compared, all m={w['m']} workers, "
+             f"tensors {','.join(_state_keys(w))}: {bad} unequal elements"
+             for variant, bad in zip(variants, unequal)]
+    lines.append(f"{name}: {time.time() - t0:.0f} s")
+    print("\n".join(lines))
     out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
     if os.path.isdir(out):
-        with open(os.path.join(out, f"fullp_{name}_{variant}.txt"), "w") as f:
-            f.write(line + "\n")
-    assert compared == w["P"] and unequal == 0, line
-    _free(s)
+        with open(os.path.join(out, f"fullp_{name}.txt"), "w") as f:
+            f.write("\n".join(lines) + "\n")
+    assert compared == w["P"] and not any(unequal), lines
+    for s in runs:
+        _free(s)
 
 
 # ------------------------------------------------------------------ seeded random configurations
