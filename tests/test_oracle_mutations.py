@@ -28,6 +28,17 @@ MUTATIONS = [
      "case 1: *cos_out = sin_psi; *sin_out = cos_psi;  break;", NOISE),                                        # quadrant sign
     ("slowmo_noise.c", "s ^= s >> 27;", "s ^= s >> 28;", NOISE),                                               # hash shift
     ("slowmo_noise.c", "return z[j & 1];", "return z[0];", NOISE),                                             # sine output never used
+    ("slowmo_oracle.c", "pow_b1 = pow_b2 = 1.0;", ";", PINS),                                                   # reset policy keeps the old bias-correction powers
+    ("slowmo_oracle.c", "sv = sv + v[i];", "sv = sv + h[i];", PINS),                                            # averaged second moment takes the wrong buffer
+    ("slowmo_oracle.c", "const real hbar = sh / (real)m, vbar = sv / (real)m;", "const real hbar = sh, vbar = sv;", PINS),  # buffer sums not divided
+    ("slowmo_oracle.c", "h[i] = FMA(b1, h[i], omb1 * g);", "h[i] = FMA(b1, h[i], g);", PINS),                   # (1 - beta_1) forgotten
+    ("slowmo_oracle.c", "v[i] = FMA(b2, v[i], omb2 * (g * g));", "v[i] = FMA(b2, v[i], omb2 * g);", PINS),      # gradient not squared
+    ("slowmo_oracle.c", "if (cfg->weight_decay != 0.0f) g = FMA((real)cfg->weight_decay, x, g);",
+     "if (cfg->weight_decay != 0.0f) g = FMA((real)cfg->weight_decay, g, g);", PINS),                           # L2 term on the gradient instead of x
+    ("slowmo_oracle.c", "const double gam_d = (double)(gamma_t ? gamma_t[t] : cfg->gamma);",
+     "const double gam_d = (double)cfg->gamma;", PINS),                                                        # learning-rate schedule ignored
+    ("slowmo_oracle.c", "for (uint32_t r = m - 1; r > 0; r >>= 1) nq += 1;", "for (uint32_t r = m; r > 0; r >>= 1) nq += 1;", SGP),  # one hop distance too many when m is a power of two
+    ("slowmo_noise.c", "float radius = sqrtf(-2.0f * ln_unit24(k1 + 1));", "float radius = sqrtf(-2.0f * ln_unit24(k1 + 2));", NOISE),  # u1 off by one step
     # slips that exist in the binary32 build only (the binary64 pins cannot see them)
     ("slowmo_oracle.c", "#define SQRT(a) sqrtf(a)", "#define SQRT(a) sqrtf(sqrtf(a))", F32),                    # wrong root in the float build
     ("slowmo_oracle.c", "#define FMA(a, b, c) fmaf((a), (b), (c))", "#define FMA(a, b, c) fmaf((a), (b), (float)(int)(c))", F32),  # a cast that truncates
