@@ -36,6 +36,7 @@ UNIT = "updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 HEADLINE = "stress_tau12"
+E2E_CHUNKS = 16
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -547,14 +548,14 @@ def run_ours(args):
             s.synchronize()
             host_in.copy_(s.grad.view(w["m"], s.pitch)[:, :w["P"]])
         e2e_steps = max(1, min(args.steps, 4))
-        e2e_ms = time_steps_e2e(s, w, e2e_steps, 1, host_in, host_out)
+        e2e_ms = time_steps_e2e(s, w, e2e_steps, 1, host_in, host_out, args.e2e_chunks)
         e2e_value, _ = aggregate_throughput(w["m"] * w["P"] * w["tau"] * e2e_steps, e2e_ms, dev)
         e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": host_in.numel() * 4,
                "d2h_bytes_per_step": host_out.numel() * 4, "steps": e2e_steps,
                "ms_per_step": round(e2e_ms / e2e_steps, 3),
                "note": "each step is one slowmo_iteration_host%s call: uploads the per-worker %s [m,P] from pinned "
-                       "host memory and reads x_{t+1,0} back, pipelined with the kernels over 16 column windows"
-                       % ("" if generated else "_supplied", "centres c" if generated else "gradient G")}
+                       "host memory and reads x_{t+1,0} back, pipelined with the kernels over %d column windows"
+                       % ("" if generated else "_supplied", "centres c" if generated else "gradient G", args.e2e_chunks)}
         del host_in, host_out
     release(s)
 
@@ -737,6 +738,8 @@ def main():
     ap.add_argument("--no-average", action="store_true",
                     help="run the workload without the exact average (Section 6 of the paper)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end measurement")
+    ap.add_argument("--e2e-chunks", type=int, default=E2E_CHUNKS,
+                    help="column windows the end-to-end call pipelines its copies and kernels over")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the direct-variant figure of the same workload and the other workloads")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
