@@ -36,7 +36,7 @@ UNIT = "updates/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 HEADLINE = "stress_tau12"
-E2E_CHUNKS = 16
+E2E_CHUNKS = 64
 
 
 # ----------------------------------------------------------------------------- bytes and peaks
@@ -332,7 +332,7 @@ def time_steps(s, w, steps, warmup, grad=None, fused=False, lazy=False):
     return total, local, outer, first
 
 
-def time_steps_e2e(s, w, steps, warmup, host_in, host_out, chunks=16):
+def time_steps_e2e(s, w, steps, warmup, host_in, host_out, chunks=E2E_CHUNKS):
     """The same step through the C ABI with host buffers: every step uploads that step's
     per-worker input data from pinned host memory and reads the new anchor back."""
     import torch

@@ -198,7 +198,7 @@ __device__ __forceinline__ uint64_t noise_counter(uint64_t vec_index) { return k
 // arithmetic, used by the kernels that wait on HBM anyway (there the shorter instruction stream
 // measured 0.4-2 % slower). true: the two-word packed map and packed arithmetic (about a quarter
 // fewer instructions per update), used by the kernels that are bound by instruction issue: the
-// virtual-replica first step and the outer step with the last inner step fused in.
+// virtual-replica first step, the outer step with the last inner step fused in, and the SGP step.
 template <bool PACKED>
 __device__ __forceinline__ float4 generated_gradient(uint64_t key, uint64_t counter, const float4 &a, const float4 &x,
                                                      const float4 &c, float sigma) {

@@ -843,8 +843,11 @@ def test_largest_parameter_count_the_library_accepts(grad_mode, m, variant, layo
     # P = 2^32 - 4096 is the largest vector slowmo_create takes (columns are indexed with 32 bits):
     # rows of 17 GB, 100-140 GB of state. Compared with the oracle at both ends, around the columns whose
     # byte offsets pass 2^32 and 2^33, in the last tiles, and on sampled coordinates.
+    import gc
     import torch
     P = 2**32 - 4096
+    gc.collect()
+    torch.cuda.empty_cache()          # memory cached from earlier tests counts as free
     free, _ = torch.cuda.mem_get_info()
     need = 4 * P * ((3 * m + 3) if grad_mode == "generated" else (3 * m + 2)) + (8 << 30)
     if free < need:
