@@ -901,8 +901,8 @@ def test_every_coordinate_of_a_full_size_workload(name, variants):
     """Selected with -m fullp only (minutes of oracle time per workload). Every named variant runs the
     whole workload on the GPU; then the oracle goes over the vector once, in chunks of 2^22 coordinates,
     and every element of every state tensor of every variant is compared with it bit for bit. The count
-    of coordinates compared and of unequal elements is printed (run with -s) and written to
-    gpurun_out/fullp_<name>.txt when that folder exists."""
+    of coordinates compared and of unequal elements is printed (run with -s) and, when the environment
+    variable SLOWMO_FULLP_OUT names a folder, written to fullp_<name>.txt there."""
     import os
     import time
     w = workloads.workload(name)
@@ -932,8 +932,8 @@ def test_every_coordinate_of_a_full_size_workload(name, variants):
              for variant, bad in zip(variants, unequal)]
     lines.append(f"{name}: {time.time() - t0:.0f} s")
     print("\n".join(lines))
-    out = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
-    if os.path.isdir(out):
+    out = os.environ.get("SLOWMO_FULLP_OUT", "")
+    if out and os.path.isdir(out):
         with open(os.path.join(out, f"fullp_{name}.txt"), "w") as f:
             f.write("\n".join(lines) + "\n")
     assert compared == w["P"] and not any(unequal), lines
