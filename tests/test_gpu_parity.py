@@ -960,13 +960,18 @@ def _random_case(rng):
                 x_init=float(rng.choice([0.0, -0.5])), no_average=no_average)
 
 
-@pytest.mark.parametrize("case", range(48))
+@pytest.mark.parametrize("case", range(72))
 def test_seeded_random_configurations_match_the_oracle(case):
     rng = np.random.Generator(np.random.PCG64(1000 + case))
     w = _random_case(rng)
     variant = str(rng.choice(["direct", "staged", "fused", "lazy"]))
+    layout = "default"
+    if case >= 48:   # more workers than noise keys fit the kernel arguments, either local-step layout
+        w.update(m=int(rng.choice([65, 96, 130])), P=int(rng.integers(1, 1500)))
+        layout = str(rng.choice(["default", "row_tiles", "column_owner"]))
     s = _slowmo(w, guard=64)
     s.set_variant("outer", variant)
+    s.set_variant("local", layout)
     grad = None
     if w["grad_mode"] == "supplied":
         grad = s.alloc_gradient()
