@@ -26,6 +26,9 @@
  *   Errors     Every call returns a SLOWMO_* status; nothing aborts or throws. CUDA
  *              failures are sticky in the context (SLOWMO_ECUDA; the cudaError_t is
  *              available from slowmo_last_cuda_error).
+ *   Tracing    slowmo_local_steps, slowmo_outer_step, slowmo_iteration_host*, slowmo_materialize
+ *              and slowmo_outer_step_sharded each open an NVTX range of their own name for the
+ *              duration of the call (a no-op unless a profiler is attached).
  *   Numerics   All arithmetic is IEEE binary32 with the operation order documented at each
  *              call; the same configuration and seed give bit-identical state on every run.
  */
