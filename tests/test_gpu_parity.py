@@ -536,6 +536,29 @@ def test_call_order_and_argument_errors():
     s.close()
 
 
+def test_empty_requests_are_accepted_and_change_nothing():
+    # zero inner steps, zero columns, zero noise draws: legal no-ops at any point of the loop
+    import torch
+    w = workloads.workload("tiny", P=37, m=3)
+    s = _slowmo(w, guard=64)
+    s.local_steps(2)
+    before = {k: s.get_params(k).copy() for k in _state_keys(w)}
+    s.local_steps(0)
+    assert s.counters() == (0, 2, 2)
+    assert s.get_params("x", offset=37, count=0).shape == (3, 0)
+    assert s.get_params("anchor", offset=5, count=0).shape == (1, 0)
+    s.set_params("u", np.zeros(1, np.float32), offset=0, count=0)
+    s.debug_noise(3, 0, 0, 0, 0, 0)
+    for k in _state_keys(w):
+        assert np.array_equal(before[k].view(np.uint32), s.get_params(k).view(np.uint32)), k
+    s.local_steps(w["tau"] - 2)
+    s.outer_step()
+    s.run(w["T"] - 1)
+    _check_against_oracle(s, w, np.arange(w["P"]), exact=True)
+    assert s.guards_intact()
+    s.close()
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_survives():
     from paper_1910_00643_b200 import SlowMoError, binding
     w = workloads.workload("tiny", P=3000)
