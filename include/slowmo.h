@@ -43,6 +43,9 @@ extern "C" {
 
 typedef struct slowmo_ctx slowmo_ctx;
 
+/* Largest parameter count per replica: the kernels index 4-column groups with 32 bits. */
+#define SLOWMO_MAX_P ((1ull << 34) - 16384)
+
 enum {
   SLOWMO_OK = 0,
   SLOWMO_EINVAL = -1,   /* bad argument (value, enum, NULL)                         */
@@ -103,7 +106,7 @@ enum {
  * hash at creation.
  */
 typedef struct {
-  uint64_t P;   /* parameters per replica (> 0)                                  */
+  uint64_t P;   /* parameters per replica (> 0, <= SLOWMO_MAX_P)                 */
   uint32_t m;   /* workers / replicas (> 0)                                      */
   uint32_t tau; /* base-optimizer steps per outer iteration (> 0)                */
   float alpha;  /* slow learning rate (> 0)                                      */

@@ -133,8 +133,8 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
 
   const uint32_t tid = threadIdx.x;
   const uint32_t warp = tid >> 5;
-  const uint32_t total_cols = A.nvec * 4u;  // fits: nvec <= 2^30 is enforced by the launcher
-  const uint32_t ntiles = (total_cols + kTileCols - 1) / kTileCols;
+  const uint64_t total_cols = 4ull * A.nvec;  // beyond 2^32 for the largest vectors: column offsets are 64-bit
+  const uint32_t ntiles = (uint32_t)((total_cols + kTileCols - 1) / kTileCols);
   const uint32_t nchunks = (A.m + kStageRows - 1) / kStageRows;
   constexpr int kPasses = POLICY == 2 ? 1 + NBUF : 1;  // x, then h (and v) when averaging
 
@@ -159,8 +159,8 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
     const uint32_t lane = tid & 31u;
     uint32_t job = 0, issued = 0;  // issued: jobs whose copies were started
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-      const uint32_t col0 = tile * kTileCols;
-      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      const uint64_t col0 = (uint64_t)tile * kTileCols;
+      const uint32_t ncols = (uint32_t)min((uint64_t)kTileCols, total_cols - col0);
       for (int pass = 0; pass < kPasses; ++pass) {
         const float *src = pass == 0 ? A.x : (pass == 1 ? A.h : A.v);
         for (uint32_t c = 0; c < nchunks; ++c, ++job) {
@@ -191,8 +191,8 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
     // thread tid owns the column groups tid + k*kConsumerThreads (k < kSub) of the tile
     uint32_t job = 0, outs = 0;
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-      const uint32_t col0 = tile * kTileCols;
-      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      const uint64_t col0 = (uint64_t)tile * kTileCols;
+      const uint32_t ncols = (uint32_t)min((uint64_t)kTileCols, total_cols - col0);
       float4 x0[kSub], u0[kSub];
 
       for (int pass = 0; pass < kPasses; ++pass) {
@@ -239,7 +239,7 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
         for (int k = 0; k < kSub; ++k) {
           const uint32_t lc = (tid + k * kConsumerThreads) * 4u;
           if (lc >= ncols) continue;
-          const uint64_t col = (uint64_t)col0 + lc;
+          const uint64_t col = col0 + lc;
           const float4 mean = make_float4(__fdiv_rn(s[k].x, A.m_float), __fdiv_rn(s[k].y, A.m_float),
                                           __fdiv_rn(s[k].z, A.m_float), __fdiv_rn(s[k].w, A.m_float));
           float4 outv = mean;  // passes 1, 2: averaged buffer
@@ -284,8 +284,8 @@ outer_step_staged_kernel(const OuterArgs A, int *status) {
     const uint32_t lane = tid & 31u;
     uint32_t outs = 0;
     for (uint32_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-      const uint32_t col0 = tile * kTileCols;
-      const uint32_t ncols = min((uint32_t)kTileCols, total_cols - col0);
+      const uint64_t col0 = (uint64_t)tile * kTileCols;
+      const uint32_t ncols = (uint32_t)min((uint64_t)kTileCols, total_cols - col0);
       for (int pass = 0; pass < kPasses; ++pass, ++outs) {
         const uint32_t ob = outs % kOutBufs, oround = outs / kOutBufs;
         if (lane == 0) mbar_wait(&S.out_full[ob], oround & 1u, &S.abort, status, 4);
@@ -341,7 +341,7 @@ inline cudaError_t outer_staged_configure() {
 
 inline void launch_outer_staged(const OuterArgs &A, int nbuf, int policy, int num_sms, int *status,
                                 cudaStream_t stream) {
-  const uint32_t ntiles = (A.nvec * 4u + kTileCols - 1) / kTileCols;
+  const uint32_t ntiles = (uint32_t)((4ull * A.nvec + kTileCols - 1) / kTileCols);
   uint32_t grid = (uint32_t)num_sms * kStagedCtasPerSm;
   if (grid > ntiles) grid = ntiles;
   const size_t bytes = sizeof(StagedSmem);

@@ -219,7 +219,7 @@ int slowmo_create(const slowmo_config *cfg, const slowmo_buffers *buf, void *cud
   if (cfg->base < SLOWMO_BASE_NESTEROV || cfg->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
   if (cfg->no_average != 0 && cfg->no_average != 1) return SLOWMO_EINVAL;
   if (cfg->no_average && cfg->buffer_policy == SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
-  if (cfg->P > (1ull << 32) - 4096) return SLOWMO_EINVAL;  // columns are indexed with 32 bits
+  if (cfg->P > SLOWMO_MAX_P) return SLOWMO_EINVAL;  // 4-column groups are indexed with 32 bits
   if (!finite_pos(cfg->alpha) || !unit_interval(cfg->beta) || !finite_pos(cfg->gamma)) return SLOWMO_EINVAL;
   if (cfg->buffer_policy < SLOWMO_BUF_RESET || cfg->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
   if (!generated && cfg->grad_mode != SLOWMO_GRAD_SUPPLIED) return SLOWMO_EINVAL;
@@ -580,7 +580,7 @@ int slowmo_outer_step_sharded(const slowmo_shard_args *a, void *cuda_stream) {
   if (a->base < SLOWMO_BASE_NESTEROV || a->base > SLOWMO_BASE_SGP_ADAM) return SLOWMO_EINVAL;
   if (a->buffer_policy < SLOWMO_BUF_RESET || a->buffer_policy > SLOWMO_BUF_AVERAGE) return SLOWMO_EINVAL;
   if (a->world == 0 || a->world > kMaxShardGpus || a->rank >= a->world || a->m_local == 0) return SLOWMO_EINVAL;
-  if (a->P == 0 || a->P > (1ull << 32) - 4096 || a->pitch < a->P) return SLOWMO_EINVAL;
+  if (a->P == 0 || a->P > SLOWMO_MAX_P || a->pitch < a->P) return SLOWMO_EINVAL;
   if (a->pitch % 4 != 0) return SLOWMO_EALIGN;
   if (!finite_pos(a->alpha) || !unit_interval(a->beta) || !finite_pos(a->gamma_t)) return SLOWMO_EINVAL;
   if (!a->x || !a->h || !a->anchor || !a->u || (adam && !a->v)) return SLOWMO_EINVAL;

@@ -67,11 +67,18 @@ def _create(binding, buf_overrides=None, **cfg_overrides):
     dict(gamma=float("nan")), dict(beta=1.0), dict(beta=-0.1), dict(alpha=0.0), dict(base=7),
     dict(buffer_policy=3), dict(grad_mode=2), dict(mu=1.0), dict(weight_decay=-1.0),
     dict(base="adam", adam_b1=1.0), dict(base="adam", adam_b2=-0.5), dict(base="adam", adam_eps=0.0),
-    dict(sigma=-1.0), dict(a_lo=2.0, a_hi=1.0), dict(P=2**33), dict(P=2**32 - 4095), dict(tensor_sizes=[4000, 97]),
+    dict(sigma=-1.0), dict(a_lo=2.0, a_hi=1.0), dict(P=2**35), dict(P=2**34 - 16383), dict(tensor_sizes=[4000, 97]),
     dict(tensor_sizes=[4096, 0]),
 ])
 def test_create_rejects_bad_configurations(binding, bad):
     assert _create(binding, **bad) == binding.EINVAL
+
+
+def test_parameter_count_limit(binding):
+    # one parameter more than SLOWMO_MAX_P is refused even when the rows are long enough
+    assert _create(binding, dict(pitch=2**34), P=2**34 - 16383) == binding.EINVAL
+    # so is a worker count whose row tiles no longer fit one grid dimension
+    assert _create(binding, dict(pitch=2**33), P=2**33, m=2**9) == binding.EINVAL
 
 
 def test_create_rejects_bad_buffers(binding):
